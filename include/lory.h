@@ -250,8 +250,9 @@ int lory_check_status(const lory_dims* dims, void* workspace, size_t workspace_b
  *
  * Limit: (S*d + S*E) * 4 bytes, S = B*L/T, must not exceed LORY_NOALLOC_SCRATCH_BYTES; larger
  * problems return LORY_ERR_TOO_LARGE and launch nothing.
- * The first call on each device looks up the array's device address (cudaGetSymbolAddress) with that
- * device current and remembers it; make that first call outside any stream capture.
+ * Every call looks up the array's device address (cudaGetSymbolAddress) for the current device and keeps no
+ * copy of it, so a context that was reset in between is harmless.  The first call on a device also loads the
+ * library's device code there: make that first call outside any stream capture.
  * All calls on one device share the one array, and it keeps the previous call's contents.  Nothing in
  * it needs clearing (every element is rewritten before it is read), but two calls whose kernels can
  * overlap on the GPU -- different streams, or different host threads -- race on it: keep calls on one
@@ -280,6 +281,24 @@ int lory_selftest_bounded_wait(const lory_dims* dims, void* workspace, size_t wo
  */
 int lory_profile_enable(int on);
 int lory_profile_read(int max_records, const char** labels, float* ms);
+
+/*
+ * Diagnostic (the paper has no counterpart): bandwidth of a write-then-read-back ring in device memory, the
+ * measurement behind the decision where the per-segment merged weights and their gradients travel between the
+ * kernel that writes them and the kernel that reads them (HBM or the L2 cache).
+ * The ring has `slots` regions of `slot_bytes` (rounded down to a whole number of 16-byte vectors per thread).
+ * Twice as many CTAs as the device has SMs each own one slice of every slot; in iteration i a CTA writes its
+ * slice of slot i mod slots (mode bit 0) and reads the slice of the CTA `shift` positions further in slot
+ * (i - lag) mod slots (mode bit 1), with loads and stores that bypass L1.  Reads hit L2 while
+ * (lag + 1) * slot_bytes still fits there.  One untimed pass fills the ring, then `iters` iterations are timed
+ * with CUDA events; the call synchronises the stream.  Bytes moved: iters * slot_bytes per active direction.
+ *   buf      DEVICE scratch, 256-byte aligned, >= slots * slot_bytes + 256 bytes
+ *   ms_out   HOST float, duration of the timed pass in milliseconds
+ * Errors: LORY_ERR_NULL, LORY_ERR_SHAPE (slots < 1, lag outside [0, slots], iters < 1, mode outside 1..3,
+ * shift < 0, slot too small), LORY_ERR_WORKSPACE (buffer too small or misaligned), LORY_ERR_CUDA.
+ */
+int lory_probe_l2_ring(void* buf, size_t buf_bytes, size_t slot_bytes, int slots, int lag, int iters, int mode,
+                       int shift, float* ms_out, void* cuda_stream);
 
 /* Number of kernel launches issued by the last forward / backward call on this thread. */
 int lory_last_launch_count(void);

@@ -59,6 +59,7 @@ _SIGNATURES = {
     "lory_route_noalloc": (ctypes.c_int, [_DP] + [_vp] * 5),
     "lory_expert_utilization": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int, _vp, _vp]),
     "lory_selftest_bounded_wait": (ctypes.c_int, [_DP, _vp, _sz, _vp]),
+    "lory_probe_l2_ring": (ctypes.c_int, [_vp, _sz, _sz] + [ctypes.c_int] * 5 + [ctypes.POINTER(ctypes.c_float), _vp]),
     "lory_profile_enable": (ctypes.c_int, [ctypes.c_int]),
     "lory_profile_read": (ctypes.c_int, [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)]),
 }
@@ -238,3 +239,11 @@ def lory_expert_utilization(route_w, counts, stream=None):
 def lory_selftest_bounded_wait(dims, workspace, stream=None):
     """Makes a bounded device-side wait expire on purpose; lory_check_status must then report the timeout."""
     _check(load().lory_selftest_bounded_wait(ctypes.byref(dims), _ptr(workspace), _nbytes(workspace), _stream(stream)))
+
+
+def lory_probe_l2_ring(buf, slot_bytes, slots, lag, iters, mode=3, shift=0, stream=None):
+    """Milliseconds of the timed pass of the write-then-read-back ring (diagnostic; see include/lory.h)."""
+    ms = ctypes.c_float(0.0)
+    _check(load().lory_probe_l2_ring(_ptr(buf), _nbytes(buf), int(slot_bytes), int(slots), int(lag), int(iters),
+                                     int(mode), int(shift), ctypes.byref(ms), _stream(stream)))
+    return ms.value

@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblory.so")
-SOURCES = ["lory_api.cu", "routing.cu", "simt.cu", "tc.cu", "noalloc.cu", "block.cu"]
+SOURCES = ["lory_api.cu", "routing.cu", "simt.cu", "tc.cu", "noalloc.cu", "block.cu", "probe.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-shared",

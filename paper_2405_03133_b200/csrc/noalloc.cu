@@ -10,22 +10,14 @@ namespace lory {
 // Every GPU that loads this library carries these 4 MiB until the process exits.
 static __device__ __align__(256) float g_route_scratch[LORY_NOALLOC_SCRATCH_BYTES / sizeof(float)];
 
-// Device address of g_route_scratch per device ordinal.  In host code the array's name only
-// stands in for the symbol; the address a kernel can use comes from cudaGetSymbolAddress,
-// asked for while that device is current.
-static const int kMaxDevices = 64;
-static float* g_scratch_addr[kMaxDevices];
-
+// In host code the array's name only stands in for the symbol; the address a kernel can use comes from
+// cudaGetSymbolAddress, asked for while the device is current.  It is asked for on every call and never kept:
+// the address belongs to the device's primary context, and a remembered copy would dangle once that context
+// has been destroyed and created again (cudaDeviceReset).  The lookup allocates nothing.
 static int scratch_for_current_device(float** out) {
-  int dev = 0;
-  LORY_CUDA_OK(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= kMaxDevices) return LORY_ERR_CUDA;
-  if (!g_scratch_addr[dev]) {
-    void* ptr = nullptr;
-    LORY_CUDA_OK(cudaGetSymbolAddress(&ptr, g_route_scratch));
-    g_scratch_addr[dev] = static_cast<float*>(ptr);
-  }
-  *out = g_scratch_addr[dev];
+  void* ptr = nullptr;
+  LORY_CUDA_OK(cudaGetSymbolAddress(&ptr, g_route_scratch));
+  *out = static_cast<float*>(ptr);
   return LORY_OK;
 }
 
