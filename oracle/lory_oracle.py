@@ -354,6 +354,48 @@ def backward_segments(x, w_r, W1, W2, W3, T, dy, seg_ids):
     return out
 
 
+def backward_every_segment(x, w_r, W1, W2, W3, T, dy, d_rows, group=8):
+    """Everything of the backward that contracts over the whole FFN-hidden dimension, for every segment
+    and without keeping the per-segment merged-weight gradients of the whole batch: the FFN-path part of
+    dx, the routing gradient dw (whole table), and, for the chosen hidden-state indices `d_rows`, the
+    slices dW2[:, d_rows, :], dW1[:, :, d_rows], dW3[:, :, d_rows] of the expert gradients
+    (dWk_e = sum_s w_{s,e} dWbar_k,s, accumulated over the segments).
+    Segments are taken `group` at a time only so that the experts are read once per group: the merge of a
+    group is the matrix product w[group] . theta (Eq. 2 for several s), dw of a group is dWbar[group] . theta^T.
+    Returns (dx_ffn [S,T,d], dw [S,E], dW2_rows [E,r,f], dW1_cols [E,f,r], dW3_cols [E,f,r])."""
+    d_rows = np.asarray(d_rows, dtype=np.int64)
+    x, dy = _f64(x), _f64(dy)
+    W1, W2, W3 = map(_f64, (W1, W2, W3))
+    B, L, d = x.shape
+    S = B * (L // T)
+    E, f, _ = W1.shape
+    _, _, w = route(x, w_r, T)
+    seg_x = x.reshape(S, T, d)
+    seg_dy = dy.reshape(S, T, d)
+    W1f, W2f, W3f = W1.reshape(E, -1), W2.reshape(E, -1), W3.reshape(E, -1)
+    dx_ffn = np.empty((S, T, d), F64)
+    dw = np.empty((S, E), F64)
+    r = len(d_rows)
+    dW2_rows = np.zeros((E, r, f), F64)
+    dW1_cols = np.zeros((E, f, r), F64)
+    dW3_cols = np.zeros((E, f, r), F64)
+    for s0 in range(0, S, group):
+        s1 = min(S, s0 + group)
+        g = s1 - s0
+        Wb1 = (w[s0:s1] @ W1f).reshape(g, f, d)
+        Wb3 = (w[s0:s1] @ W3f).reshape(g, f, d)
+        Wb2 = (w[s0:s1] @ W2f).reshape(g, d, f)
+        dWb1, dWb2, dWb3 = np.empty_like(Wb1), np.empty_like(Wb2), np.empty_like(Wb3)
+        for i in range(g):
+            dx_ffn[s0 + i], dWb1[i], dWb2[i], dWb3[i] = _segment_grads(seg_x[s0 + i], seg_dy[s0 + i], Wb1[i], Wb2[i], Wb3[i])
+        dw[s0:s1] = (dWb1.reshape(g, -1) @ W1f.T + dWb2.reshape(g, -1) @ W2f.T + dWb3.reshape(g, -1) @ W3f.T)
+        wT = np.ascontiguousarray(w[s0:s1].T)                    # [E, g]
+        dW2_rows += (wT @ dWb2[:, d_rows, :].reshape(g, -1)).reshape(E, r, f)
+        dW1_cols += (wT @ dWb1[:, :, d_rows].reshape(g, -1)).reshape(E, f, r)
+        dW3_cols += (wT @ dWb3[:, :, d_rows].reshape(g, -1)).reshape(E, f, r)
+    return dx_ffn, dw, dW2_rows, dW1_cols, dW3_cols
+
+
 # --------------------------------------------------------------------------
 # Inference (Section 3.1 "Prompt-only routing during inference"; appendix
 # "Inference Methods") and the expert-utilisation statistic (appendix

@@ -188,25 +188,19 @@ def test_first_segment_routes_itself():
         np.testing.assert_array_equal(w[b * N + 2], pr[b * N + 1])
 
 
-# ---- I14: independent autograd transcription of Algorithm 1 ----------------
-def algorithm1_torch(x, w_r, W1, W2, W3, T):
+# ---- I14: independent autograd formulation of the layer -----------------------
+def lory_layer_torch(x, w_r, W1, W2, W3, T):
+    """The layer written per sequence with torch ops: segment s of a sequence is weighted by the router
+    output of segment s-1, the first segment by its own output cut from the graph."""
     B, L, d = x.shape
-    E = w_r.shape[0]
     N = L // T
-    seg_x = x.view(B * N, T, d)
-    rep = seg_x.mean(dim=1)
-    e = torch.softmax(rep @ w_r.T, dim=-1)
-    e_first = e.view(B, N, E)[:, 0]
-    e = torch.roll(e, 1, dims=0).view(B, N, E).clone()
-    e[:, 0] = e_first.detach()
-    e = e.view(B * N, E)
-    Wb1 = torch.einsum("se,efd->sfd", e, W1)
-    Wb3 = torch.einsum("se,efd->sfd", e, W3)
-    Wb2 = torch.einsum("se,edf->sdf", e, W2)
-    g = torch.einsum("std,sfd->stf", seg_x, Wb1)
-    u = torch.einsum("std,sfd->stf", seg_x, Wb3)
-    seg_y = torch.einsum("stf,sdf->std", F.silu(g) * u, Wb2)
-    return seg_y.reshape(B, L, d), e
+    segs = x.reshape(B, N, T, d)
+    p = torch.softmax(torch.einsum("bnd,ed->bne", segs.mean(dim=2), w_r), dim=-1)
+    w = torch.cat([p[:, :1].detach(), p[:, :-1]], dim=1)
+    up = lambda Wk: torch.einsum("bntd,bne,efd->bntf", segs, w, Wk)
+    h = F.silu(up(W1)) * up(W3)
+    y = torch.einsum("bntf,bne,edf->bntd", h, w, W2)
+    return y.reshape(B, L, d), w.reshape(B * N, -1)
 
 
 @pytest.mark.parametrize("std,shape", [(0.02, dict()), (2.0, dict()), (4.0, dict(B=3, L=10, T=2, d=5, f=7, E=4)),
@@ -214,7 +208,7 @@ def algorithm1_torch(x, w_r, W1, W2, W3, T):
 def test_autograd_transcription_agrees(std, shape):
     p = rand_problem(w_r_std=std, seed=21, **shape)
     ts = {k: t64(p[k], True) for k in ("x", "w_r", "W1", "W2", "W3")}
-    y_t, e_t = algorithm1_torch(ts["x"], ts["w_r"], ts["W1"], ts["W2"], ts["W3"], p["T"])
+    y_t, e_t = lory_layer_torch(ts["x"], ts["w_r"], ts["W1"], ts["W2"], ts["W3"], p["T"])
     y, w, _ = fwd(p)
     np.testing.assert_allclose(y, y_t.detach().numpy(), rtol=1e-11, atol=1e-12)
     np.testing.assert_allclose(w, e_t.detach().numpy(), rtol=1e-13, atol=0)
@@ -409,6 +403,14 @@ def test_sampled_variants_match_full():
     for s, (dxs, dws) in bs.items():
         np.testing.assert_allclose(dxs, dx_ffn[s], rtol=1e-11, atol=1e-12)
         np.testing.assert_allclose(dws, g["d_route_w"][s], rtol=1e-11, atol=1e-12)
+    d_rows = [5, 0, 2]
+    for group in (8, 4, 1):     # one group, a ragged last group, segment by segment
+        dx_all, dw_all, dW2r, dW1c, dW3c = O.backward_every_segment(*a, p["dy"], d_rows, group=group)
+        np.testing.assert_allclose(dx_all, dx_ffn, rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(dw_all, g["d_route_w"], rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(dW2r, g["dW2"][:, d_rows, :], rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(dW1c, g["dW1"][:, :, d_rows], rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(dW3c, g["dW3"][:, :, d_rows], rtol=1e-11, atol=1e-12)
 
 
 # ---- I15: Appendix B figures --------------------------------------------------

@@ -1,6 +1,6 @@
 """GPU parity: the CUDA path through the C ABI against the CPU oracle, element by element,
 on the same seeded inputs.  Tolerances: fp32 mode max|diff|/max|ref| <= 1e-4 per tensor,
-bf16 mode <= 2e-2 per tensor."""
+bf16 mode <= 2e-2 per tensor; the routing tables are fp32 in either mode and are held to 1e-5."""
 import numpy as np
 import pytest
 
@@ -23,9 +23,12 @@ def oracle_all(wl, inp):
     return dict(y=y, route_w=w, route_p=p, **g)
 
 
+ROUTE_TOL = 1e-5   # route_w, route_p: fp32 sums and an fp32 softmax whatever the storage type
+
+
 def compare(wl, got, ref, tol, keys=None):
     errs = {k: max_rel(got[k], ref[k]) for k in (keys or ALL_KEYS)}
-    bad = {k: v for k, v in errs.items() if not v <= tol}
+    bad = {k: v for k, v in errs.items() if not v <= (min(tol, ROUTE_TOL) if k in ("route_w", "route_p") else tol)}
     assert not bad, f"{wl.name}: over tolerance {tol}: {bad} (all: {errs})"
     return errs
 
