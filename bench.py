@@ -57,9 +57,42 @@ def kernel_flops(wl):
     }
 
 
-# algorithmic HBM bytes per step of each labelled kernel (per launch for the three "wgrad" launches): inputs read
-# once + outputs written once, bf16
-def kernel_bytes(wl):
+# Which roofline bounds a labelled kernel: the dense contractions are tensor-core work, the routing-weighted sums
+# over the experts (merge, its adjoint) and the pooling stream the method's tensors through HBM.
+KERNEL_BOUND = {"gemm1_swiglu": "tensor", "gemm2": "tensor", "dh_dswiglu": "tensor", "wgrad": "tensor", "dx": "tensor",
+                "merge": "hbm", "stage2": "hbm", "pool_router": "hbm"}
+
+
+def compulsory_bytes(wl):
+    """What the method itself has to move per step: x read in the forward and in the backward, y written, dY read,
+    dX written (5 activation tensors), the experts read in the forward and in the backward and their gradients
+    written (3 passes over E * 3 * d * f parameters); bf16.  Merged weights, their gradients and saved activations
+    are choices of an implementation and are not in here."""
+    return 5 * wl.tokens * wl.d * 2 + 3 * wl.E * 3 * wl.d * wl.f * 2
+
+
+# algorithmic bytes of one launch of each labelled kernel: only tensors the method defines (x, y, dY, dX, the
+# experts, their gradients), each once.  The HBM-bound kernels are measured against these.
+def method_bytes(wl):
+    act = 2 * wl.tokens * wl.d
+    Pb = 2 * wl.d * wl.f                      # one expert matrix
+    launches_256 = (wl.S + 255) // 256
+    return {
+        "pool_router": act,                                  # x
+        "merge": 3 * wl.E * Pb,                              # the experts, once
+        "gemm1_swiglu": act,                                 # x
+        "gemm2": act,                                        # y
+        "dh_dswiglu": act,                                   # dY
+        "wgrad": 2 * wl.tokens * (wl.d + wl.f),              # per launch: its two activation operands
+        "stage2": 2 * 3 * wl.E * Pb,                         # the experts in, their gradients out
+        "dx": act,                                           # dX
+        "_launches_256": launches_256,
+    }
+
+
+# HBM bytes per step of each labelled kernel AS IMPLEMENTED (per launch for the three "wgrad" launches): inputs read
+# once + outputs written once, merged weights, their gradients and the saved activations included; bf16
+def implementation_bytes(wl):
     tok, S, d, f, E = wl.tokens, wl.S, wl.d, wl.f, wl.E
     P1 = d * f
     launches_256 = (S + 255) // 256
@@ -79,6 +112,12 @@ def kernel_bytes(wl):
         "wgrad": 2 * (tok * (d + f) + S * P1),                      # per matrix: two activations -> dWbar
         "dx": 2 * (2 * tok * f + 2 * S * P1 + tok * d),             # dG, dU, Wbar1, Wbar3 -> dx
     }
+
+
+def implementation_bytes_per_step(wl):
+    kb = implementation_bytes(wl)
+    return (kb["merge"] + kb["stage2"] + kb["gemm1_swiglu"] + kb["gemm2"] + kb["dh_dswiglu"] + 3 * kb["wgrad"]
+            + kb["dx"] + kb["pool_router"])
 
 
 # DRAM traffic of one launch (dram__bytes_read.sum + dram__bytes_write.sum) from a one-pass ncu capture of one
@@ -125,7 +164,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -242,6 +281,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the number of sequences B (profiling on a small case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the second timed region of >= 1 s")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -307,69 +347,118 @@ def main():
     lory.lory_check_status(dims, ws)
     barrier()
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    # ---- timed region: K steps, device-resident inputs, per-kernel events recorded alongside ----
-    lory.lory_profile_enable(True)
-    barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_wall0 = time.time()
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-    ev1.record()
-    barrier()
-    t_wall1 = time.time()
-    ms_total = ev0.elapsed_time(ev1)
-    records = lory.lory_profile_read()
-    lory.lory_profile_enable(False)
-    lory.lory_check_status(dims, ws)
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    def timed_region(n_steps):
+        """n_steps back to back, device-resident inputs, CUDA events on the launch stream around the whole region
+        and (through the library's profiling hooks) around every kernel; SM clocks sampled meanwhile."""
+        sampler = ClockSampler(local_rank)
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.3)
+        lory.lory_profile_enable(True)
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_wall0 = time.time()
+        ev0.record()
+        for _ in range(n_steps):
+            step()
+        ev1.record()
+        barrier()
+        t_wall1 = time.time()
+        ms = ev0.elapsed_time(ev1)
+        recs = lory.lory_profile_read()
+        lory.lory_profile_enable(False)
+        lory.lory_check_status(dims, ws)
+        return ms, recs, (sampler.stop(t_wall0, t_wall1) if rank == 0 else None)
 
+    ms_total, records, clocks = timed_region(args.steps)
     ms_per_step, value = aggregate_over_ranks(ms_total, args.steps, wl.tokens, world, dist, dev)
 
-    # ---- per-kernel statistics --------------------------------------------------------------
     peaks = load_peaks()
-    per = {}
-    for label, ms in records:
-        per.setdefault(label, []).append(ms)
-    kf, kb = kernel_flops(wl), kernel_bytes(wl)
-    kernels = {}
-    tot_kernel_ms = sum(sum(v) for v in per.values())
-    for label, v in per.items():
-        avg = sum(v) / len(v)
-        ent = {"launches_per_step": len(v) / args.steps, "avg_ms": avg, "share": sum(v) / tot_kernel_ms}
-        # flops / bytes are per step for a label (per launch for the three weight-gradient GEMMs); a label may
-        # take several launches per step (one per 256 segments for the merge and its adjoint)
-        ms_step = sum(v) / args.steps / (3.0 if label in ("wgrad", "dtheta", "dw") else 1.0)
-        if label in kf:
-            ent["tflops"] = kf[label] / (ms_step * 1e-3) / 1e12
-        if label in kb:
-            ent["gbs"] = kb[label] / (ms_step * 1e-3) / 1e9
-        kernels[label] = ent
+    # Which measured tensor peak a run is compared with: the burst figure while the SM clock stays near its maximum
+    # (a short timed region), the sustained one once the power cap has pulled the clock down (a long region).
+    def regime(clk):
+        if clk and clk.get("sm_mhz") and clk.get("sm_max_mhz") and clk["sm_mhz"] < 0.9 * clk["sm_max_mhz"]:
+            return "sustained", peaks["bf16_tflops_sustained"]
+        return "burst", peaks["bf16_tflops"]
+
+    def kernel_stats(recs, n_steps, clk):
+        """Per label: time, share, and the fraction of the roofline that bounds it (tensor peak for the
+        contractions, HBM bandwidth over the method's own bytes for the streaming kernels)."""
+        _, tensor_peak = regime(clk)
+        per = {}
+        for label, ms in recs:
+            per.setdefault(label, []).append(ms)
+        kf, mb, ib = kernel_flops(wl), method_bytes(wl), implementation_bytes(wl)
+        tot = sum(sum(v) for v in per.values())
+        out = {}
+        for label, v in per.items():
+            avg = sum(v) / len(v)
+            ent = {"launches_per_step": len(v) / n_steps, "avg_ms": avg, "share": sum(v) / tot}
+            if clk and clk.get("sm_mhz"):
+                ent["ms_x_mhz"] = avg * clk["sm_mhz"]       # constant over clocks for a kernel bound on the SMs
+            # flops / bytes are per step for a label (per launch for the three weight-gradient GEMMs); a label may
+            # take several launches per step (one per 256 segments for the merge and its adjoint)
+            t_step = sum(v) / n_steps / (3.0 if label == "wgrad" else 1.0) * 1e-3
+            bound = KERNEL_BOUND.get(label)
+            if label in kf:
+                ent["tflops"] = kf[label] / t_step / 1e12
+            if label in mb:
+                ent["algorithmic_gbs"] = mb[label] / t_step / 1e9
+            if label in ib:
+                ent["implementation_gbs"] = ib[label] / t_step / 1e9
+            if bound == "tensor":
+                ent.update(bound="tensor", frac=ent["tflops"] / tensor_peak)
+            elif bound == "hbm":
+                ent.update(bound="hbm", frac=ent["algorithmic_gbs"] / peaks["hbm_gbs"])
+            out[label] = ent
+        return out
+
+    kernels = kernel_stats(records, args.steps, clocks)
+    reg_name, tensor_peak = regime(clocks)
     top = max(kernels, key=lambda k: kernels[k]["share"]) if kernels else None
     roofline = None
-    if top is not None:
-        # the bound of a kernel is the slower of its algorithmic flops at the tensor peak and its algorithmic
-        # bytes at the HBM peak; `achieved` and `peak` are in the unit of that bound
+    if top is not None and kernels[top].get("bound"):
         e = kernels[top]
-        t_tensor = kf.get(top, 0.0) / (peaks["bf16_tflops_sustained"] * 1e12)
-        t_hbm = kb.get(top, 0.0) / (peaks["hbm_gbs"] * 1e9)
-        if t_hbm >= t_tensor and "gbs" in e:
-            roofline = {"kernel": top, "bound": "hbm", "achieved": e["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": e["gbs"] / peaks["hbm_gbs"], "traffic": measured_traffic(wl.name, top),
-                        "peak_source": peaks["source"]}
-        elif "tflops" in e:
-            roofline = {"kernel": top, "bound": "tensor", "achieved": e["tflops"], "peak": peaks["bf16_tflops_sustained"],
-                        "unit": "TFLOP/s", "frac": e["tflops"] / peaks["bf16_tflops_sustained"],
-                        "traffic": measured_traffic(wl.name, top),
-                        "peak_source": peaks["source"] + " (sustained: timed inside a long step)"}
-    layer_tflops = flops_per_step(wl) / (ms_per_step * 1e-3) / 1e12
-    layer = {"algorithmic_tflop_per_step": flops_per_step(wl) / 1e12, "achieved_tflops": layer_tflops,
+        traffic = measured_traffic(wl.name, top)
+        alg_bytes = method_bytes(wl).get(top)
+        roofline = {"kernel": top, "bound": e["bound"], "frac": e["frac"], "traffic": traffic,
+                    "algorithmic_bytes": alg_bytes,
+                    "traffic_ratio": (traffic / alg_bytes) if (traffic and alg_bytes) else None}
+        if e["bound"] == "tensor":
+            roofline.update(achieved=e["tflops"], peak=tensor_peak, unit="TFLOP/s",
+                            peak_source=f"{peaks['source']} ({reg_name})")
+        else:
+            roofline.update(achieved=e["algorithmic_gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
+                            peak_source=peaks["source"])
+    # the whole layer: Appendix B's flop count over the step time, against the slower of flops at the tensor peak
+    # and compulsory bytes at the copy bandwidth
+    F, CB = flops_per_step(wl), compulsory_bytes(wl)
+    t_roof = max(F / (tensor_peak * 1e12), CB / (peaks["hbm_gbs"] * 1e9))
+    layer_tflops = F / (ms_per_step * 1e-3) / 1e12
+    step_traffic = None
+    ent = NCU_TRAFFIC.get(wl.name)
+    if ent is not None and ent["sources_sha1"] == cuda_sources_sha1():
+        step_traffic = sum(b * (3 if k == "wgrad" else 1) for k, b in ent["bytes"].items())
+    layer = {"algorithmic_tflop_per_step": F / 1e12, "achieved_tflops": layer_tflops,
+             "frac": t_roof / (ms_per_step * 1e-3), "frac_peak": f"{reg_name} bf16 peak, {peaks['source']}",
              "frac_of_burst_peak": layer_tflops / peaks["bf16_tflops"],
-             "frac_of_sustained_peak": layer_tflops / peaks["bf16_tflops_sustained"]}
+             "frac_of_sustained_peak": layer_tflops / peaks["bf16_tflops_sustained"],
+             "compulsory_bytes": CB, "implementation_bytes": implementation_bytes_per_step(wl),
+             "traffic": step_traffic, "traffic_ratio": (step_traffic / CB) if step_traffic else None}
+
+    # ---- the same step held for at least a second: the power cap pulls the SM clock down ----
+    sustained = None
+    if not args.no_sustained:
+        n_long = max(400, int(1.2e3 / ms_per_step))
+        ms_long, rec_long, clk_long = timed_region(n_long)
+        ms_step_long, value_long = aggregate_over_ranks(ms_long, n_long, wl.tokens, world, dist, dev)
+        tf_long = F / (ms_step_long * 1e-3) / 1e12
+        k_long = kernel_stats(rec_long, n_long, clk_long)
+        sustained = {"steps": n_long, "ms_per_step": ms_step_long, "value": value_long, "unit": UNIT,
+                     "clocks": clk_long, "achieved_tflops": tf_long,
+                     "frac_of_sustained_peak": tf_long / peaks["bf16_tflops_sustained"],
+                     "kernels": {k: {kk: v[kk] for kk in ("avg_ms", "ms_x_mhz", "frac") if kk in v}
+                                 for k, v in k_long.items()}}
 
     if rank != 0:
         if dist is not None:
@@ -448,7 +537,7 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic", "config": workload_config(wl), "clocks": clocks, "e2e": e2e,
         "gpu_launches": launches[0] * args.steps, "roofline": roofline, "cpu_baseline": cpu, "layer": layer,
-        "kernels": kernels,
+        "sustained": sustained, "kernels": kernels,
     }
     print(json.dumps(out))
     if dist is not None:

@@ -22,6 +22,8 @@ void note_cuda_error(cudaError_t e, const char* what) {
   snprintf(s.cuda_error, sizeof(s.cuda_error), "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
 }
 
+static const int kMaxDevices = 64;  // per-device host state (streams, events) is kept per device ordinal
+
 // ---- per-launch timing ---------------------------------------------------------------------
 static const int PROF_MAX = 8192;
 struct Prof {
@@ -500,9 +502,18 @@ int lory_moe_step_host(const lory_dims* dims, const void* x_host, const void* dy
   float* rw_d = (float*)(a + 4 * act);
   char* ws = a + 4 * act + rw;
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  // A second stream carries dY in while the forward runs and y out while the backward runs.
-  static thread_local cudaStream_t side = nullptr;
-  static thread_local cudaEvent_t ev_x = nullptr, ev_dy = nullptr, ev_fwd = nullptr, ev_y = nullptr;
+  // A second stream carries dY in while the forward runs and y out while the backward runs (one per host thread
+  // and device: streams and events belong to the device that was current when they were created).
+  struct Side {
+    cudaStream_t side;
+    cudaEvent_t ev_x, ev_dy, ev_fwd, ev_y;
+  };
+  static thread_local Side sides[kMaxDevices] = {};
+  int dev = 0;
+  LORY_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return LORY_ERR_CUDA;
+  cudaStream_t& side = sides[dev].side;
+  cudaEvent_t &ev_x = sides[dev].ev_x, &ev_dy = sides[dev].ev_dy, &ev_fwd = sides[dev].ev_fwd, &ev_y = sides[dev].ev_y;
   if (!side) {
     LORY_CUDA_OK(cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking));
     LORY_CUDA_OK(cudaEventCreateWithFlags(&ev_x, cudaEventDisableTiming));
@@ -651,9 +662,12 @@ struct HostPipe {
   cudaEvent_t x_in[2] = {}, dy_in[2] = {}, fwd[2] = {}, bwd[2] = {}, landed[2] = {};
   bool used[2] = {false, false};
 };
-HostPipe& host_pipe() {
-  static thread_local HostPipe hp;
-  return hp;
+// One pipeline per host thread and device.
+HostPipe* host_pipe() {
+  static thread_local HostPipe hp[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  return &hp[dev];
 }
 int host_pipe_init(HostPipe& hp) {
   if (hp.in) return LORY_OK;
@@ -694,7 +708,9 @@ int lory_moe_step_host_enqueue(const lory_dims* dims, int slot, const void* x_ho
   lory_moe_step_host_pipeline_bytes(dims, &need);
   s = check_ws(arena, arena_bytes, need);
   if (s != LORY_OK) return s;
-  HostPipe& hp = host_pipe();
+  HostPipe* hpp = host_pipe();
+  if (!hpp) return LORY_ERR_CUDA;
+  HostPipe& hp = *hpp;
   s = host_pipe_init(hp);
   if (s != LORY_OK) return s;
   Layout Lo = make_layout(*dims);
@@ -746,7 +762,9 @@ int lory_moe_step_host_enqueue(const lory_dims* dims, int slot, const void* x_ho
 
 int lory_moe_step_host_wait(int slot) {
   if (slot != 0 && slot != 1) return LORY_ERR_SHAPE;
-  HostPipe& hp = host_pipe();
+  HostPipe* hpp = host_pipe();
+  if (!hpp) return LORY_ERR_CUDA;
+  HostPipe& hp = *hpp;
   if (!hp.in || !hp.used[slot]) return LORY_OK;  // nothing was enqueued on this slot
   LORY_CUDA_OK(cudaEventSynchronize(hp.landed[slot]));
   return LORY_OK;

@@ -104,15 +104,34 @@ static int make_expert_map(CUtensorMap* m, const void* base, int R, int C, int E
   return make_map_nd(m, base, 3, dims, strides, box);
 }
 
+// Per-device state is kept per device ordinal: a process may drive several GPUs.
+static const int kMaxDevices = 64;
+static int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+  return dev;
+}
+
 static int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
+  static int n[kMaxDevices];
+  const int dev = current_device();
+  if (!n[dev]) {
+    if (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0)
+      n[dev] = 148;
   }
-  return n;
+  return n[dev];
+}
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize belongs to the (function, device) pair: set it once on every
+// device that launches the kernel.
+template <typename K>
+static int allow_dynamic_smem(K kern, int bytes, bool (&done)[kMaxDevices]) {
+  const int dev = current_device();
+  if (!done[dev]) {
+    LORY_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    done[dev] = true;
+  }
+  return LORY_OK;
 }
 
 static const int kMaxSmem = 227 * 1024 - 512;  // dynamic shared memory we may ask for (static use is < 512 B)
@@ -130,11 +149,8 @@ static int launch_tc(const char* label, const CUtensorMap& a0, const CUtensorMap
   if (tiles <= 0) return LORY_OK;
   if (tiles > 0x7fffffffL) return LORY_ERR_SHAPE;
   auto kern = tc_gemm_kernel<A_MN, B_MN, BN, MODE, EPI, B_BLK, C_BLK, CTAS>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    LORY_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile::SMEM_BYTES));
-    attr_set = true;
-  }
+  static bool attr_set[kMaxDevices];
+  LORY_TRY(allow_dynamic_smem(kern, Tile::SMEM_BYTES, attr_set));
   const int slots = sm_count() / CTAS;  // persistent CTAs (or CTA pairs)
   const int grid = CTAS * (int)(tiles < slots ? tiles : slots);
   const CUtensorMap& me0 = e0 ? *e0 : c0;
@@ -272,11 +288,8 @@ static int launch_merge(const lory_dims& D, const WsPtrs& q, const bf16* const s
   if (p.stages > 8) p.stages = 8;
   if (p.stages < 2) return LORY_ERR_SHAPE;
   const int smem = fixed + p.stages * p.stage_bytes;
-  static bool attr_set = false;
-  if (!attr_set) {
-    LORY_CUDA_OK(cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
-    attr_set = true;
-  }
+  static bool attr_set[kMaxDevices];
+  LORY_TRY(allow_dynamic_smem(merge_kernel, kMaxSmem, attr_set));
   const int grid = p.tile_end[2] < sm_count() ? p.tile_end[2] : sm_count();
   // one launch per 256 segments (each re-reads the experts once: the same ratio as one launch at S = 256)
   for (int base = 0; base < S; base += 256) {
@@ -331,12 +344,9 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const bf16* const 
   if (p.stages > 8) p.stages = 8;
   if (p.stages < 2) return LORY_ERR_SHAPE;
   const int smem = fixed + p.stages * p.stage_bytes;
-  static bool attr_set = false;
-  if (!attr_set) {
-    LORY_CUDA_OK(cudaFuncSetAttribute(stage2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
-    LORY_CUDA_OK(cudaFuncSetAttribute(stage2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
-    attr_set = true;
-  }
+  static bool attr_set[2][kMaxDevices];
+  LORY_TRY(allow_dynamic_smem(stage2_kernel<false>, kMaxSmem, attr_set[0]));
+  LORY_TRY(allow_dynamic_smem(stage2_kernel<true>, kMaxSmem, attr_set[1]));
   // One launch per 256 segments; launches after the first add to the expert gradients the earlier ones stored
   // (the same read-add-store as gradient accumulation), and each writes its own rows of the dw slabs.
   for (int base = 0; base < S; base += 256) {

@@ -163,7 +163,10 @@ class LoryPromptRoutedFFN:
         x_prompt = x_prompt.contiguous()
         y = torch.empty_like(x_prompt)
         self.route_w = torch.empty((B, E), dtype=torch.float32, device=x_prompt.device)
-        _lory.lory_moe_forward(dims, x_prompt, m.w_r, m.W1, m.W2, m.W3, y, self.route_w, None, self.ws)
+        # on the stream torch is issuing this tensor's work on, so that the call is ordered with its producers and
+        # consumers (and with later decode() calls, which share the cached workspace)
+        _lory.lory_moe_forward(dims, x_prompt, m.w_r, m.W1, m.W2, m.W3, y, self.route_w, None, self.ws,
+                               torch.cuda.current_stream(x_prompt.device))
         return y
 
     @torch.no_grad()
@@ -181,5 +184,5 @@ class LoryPromptRoutedFFN:
             raise ValueError("more new tokens per sequence than the prompt had: the cached workspace is too small")
         x_new = x_new.contiguous()
         y = torch.empty_like(x_new)
-        _lory.lory_moe_ffn(dims, x_new, None, m.W1, m.W2, m.W3, y, self.ws)
+        _lory.lory_moe_ffn(dims, x_new, None, m.W1, m.W2, m.W3, y, self.ws, torch.cuda.current_stream(x_new.device))
         return y

@@ -29,9 +29,27 @@ def test_gemm_flops_add_up_to_the_ffn_part_of_the_layer():
     assert ffn + kf["merge"] + kf["stage2"] == bench.flops_per_step(wl)
 
 
-def test_kernel_bytes_at_c3():
+def test_compulsory_bytes_at_c3():
+    """What the method has to move: five activation tensors and three passes over the experts."""
     wl = CONFIGS["C3"]
-    kb = bench.kernel_bytes(wl)
+    act = wl.tokens * wl.d * 2
+    experts = wl.E * 3 * wl.d * wl.f * 2
+    assert act == 67108864 and experts == 541065216
+    assert bench.compulsory_bytes(wl) == 5 * act + 3 * experts
+    assert 1.95e9 < bench.compulsory_bytes(wl) < 1.97e9
+    # the parts of it each kernel touches add up to the whole: x twice more in the weight-gradient GEMMs and once
+    # in the pooling on top of the five tensors, the experts three times
+    mb = bench.method_bytes(wl)
+    assert mb["merge"] == experts and mb["stage2"] == 2 * experts
+    assert mb["gemm1_swiglu"] == mb["gemm2"] == mb["dh_dswiglu"] == mb["dx"] == mb["pool_router"] == act
+    assert mb["wgrad"] == 2 * wl.tokens * (wl.d + wl.f)
+
+
+def test_implementation_bytes_at_c3():
+    """What this implementation moves on top: merged weights written once and read twice, their gradients written
+    and read, the saved activations."""
+    wl = CONFIGS["C3"]
+    kb = bench.implementation_bytes(wl)
     P1 = wl.d * wl.f * 2                       # one bf16 matrix
     act_d, act_f = wl.tokens * wl.d * 2, wl.tokens * wl.f * 2
     assert kb["merge"] == 3 * (wl.E * P1 + wl.S * P1)
@@ -41,19 +59,24 @@ def test_kernel_bytes_at_c3():
     assert kb["dh_dswiglu"] == act_d + wl.S * P1 + 4 * act_f
     assert kb["wgrad"] == act_d + act_f + wl.S * P1
     assert kb["dx"] == 2 * act_f + 2 * wl.S * P1 + act_d
-    # the whole step: W-bar written once and read twice, dW-bar written and read, experts read twice and written once
-    total = (kb["merge"] + kb["stage2"] + kb["gemm1_swiglu"] + kb["gemm2"] + kb["dh_dswiglu"] + 3 * kb["wgrad"]
-             + kb["dx"] + kb["pool_router"])
-    assert 15.0e9 < total < 15.4e9
+    assert 15.0e9 < bench.implementation_bytes_per_step(wl) < 15.4e9
+    assert 7.5 < bench.implementation_bytes_per_step(wl) / bench.compulsory_bytes(wl) < 7.9
+
+
+def test_contractions_are_tensor_bound_and_streaming_kernels_hbm_bound():
+    for k in ("gemm1_swiglu", "gemm2", "dh_dswiglu", "wgrad", "dx"):
+        assert bench.KERNEL_BOUND[k] == "tensor"
+    for k in ("merge", "stage2", "pool_router"):
+        assert bench.KERNEL_BOUND[k] == "hbm"
 
 
 def test_more_than_256_segments_cost_extra_expert_passes():
     wl = CONFIGS["C3"].with_(B=32)             # 512 segments: two launches of the merge and of its adjoint
     small = CONFIGS["C3"]
     P1 = wl.d * wl.f * 2
-    assert bench.kernel_bytes(wl)["merge"] == 3 * (2 * wl.E * P1 + wl.S * P1)
-    assert bench.kernel_bytes(wl)["stage2"] == 3 * (wl.S * P1 + 5 * wl.E * P1)
-    assert bench.kernel_bytes(small)["merge"] == 3 * (small.E * P1 + small.S * P1)
+    assert bench.implementation_bytes(wl)["merge"] == 3 * (2 * wl.E * P1 + wl.S * P1)
+    assert bench.implementation_bytes(wl)["stage2"] == 3 * (wl.S * P1 + 5 * wl.E * P1)
+    assert bench.implementation_bytes(small)["merge"] == 3 * (small.E * P1 + small.S * P1)
 
 
 def test_traffic_table_is_guarded_by_the_source_digest(monkeypatch):

@@ -107,3 +107,31 @@ def test_prompt_routed_ffn_helper():
     assert max_rel(y_prompt.double().cpu().numpy(), ref_prompt) <= TOL["bf16"]
     assert max_rel(y_new.double().cpu().numpy(), ref_new) <= TOL["bf16"]
     assert max_rel(ffn.route_w.double().cpu().numpy(), w_ref) <= 1e-5
+
+
+def test_prompt_routed_ffn_on_a_side_stream():
+    """prefill and decode issued inside `with torch.cuda.stream(s)`: inputs are produced and outputs consumed on
+    that stream only, so the library calls must run there too."""
+    from paper_2405_03133_b200.layer import LoryPromptRoutedFFN
+    from paper_2405_03133_b200.workloads import round_to_bf16
+    wl = Workload("module_prompt_stream", B=2, L=256, T=256, d=128, f=200, E=5, dtype="bf16", w_r_std=2.0, seed=69)
+    inp = make_inputs(wl)
+    m = module_for(wl, inp)
+    ffn = LoryPromptRoutedFFN(m)
+    x_new = round_to_bf16(np.random.default_rng(70).standard_normal((wl.B, 3, wl.d)).astype(np.float32))
+    xp_host = torch.from_numpy(inp["x"]).to(torch.bfloat16).pin_memory()
+    xn_host = torch.from_numpy(x_new).to(torch.bfloat16).pin_memory()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        # the inputs reach the device on the side stream, right in front of the calls that read them
+        xp = xp_host.to("cuda", non_blocking=True)
+        xn = xn_host.to("cuda", non_blocking=True)
+        y_prompt = ffn.prefill(xp)
+        y_new = ffn.decode(xn)
+        yp_host = y_prompt.to("cpu", non_blocking=True)
+        yn_host = y_new.to("cpu", non_blocking=True)
+    side.synchronize()
+    ref_prompt, ref_new, _ = O.prompt_only_inference(inp["x"], x_new, inp["w_r"], inp["W1"], inp["W2"], inp["W3"])
+    assert max_rel(yp_host.double().numpy(), ref_prompt) <= TOL["bf16"]
+    assert max_rel(yn_host.double().numpy(), ref_new) <= TOL["bf16"]
