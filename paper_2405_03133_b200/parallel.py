@@ -107,11 +107,24 @@ def cuda_layer_fns(B: int, L: int, T: int, dtype: str = "bf16", flags: int = 0):
     return run_forward, run_backward
 
 
-def torch_all_reduce(group=None):
-    """all_reduce callable over torch.distributed (NCCL on GPUs, gloo on CPU): sum, in place."""
+def torch_all_reduce(group=None, accumulate_in_fp32: bool = True):
+    """all_reduce callable over torch.distributed (NCCL on GPUs, gloo on CPU): sum, in place.
+
+    The partial y and dx of the slices are bf16 tensors in bf16 mode.  Summed as they are, a ring or tree of R
+    ranks rounds the running sum to bf16 up to R - 1 times, on top of the rounding each slice already carries.
+    With accumulate_in_fp32 (the default) a 16-bit tensor is widened to fp32, all-reduced, and rounded ONCE on
+    the way back: twice the bytes on the wire for the small activation tensors (never for weights, which are
+    not exchanged), and a result that does not depend on the number of ranks or on the reduction order beyond
+    fp32 rounding."""
+    import torch
     import torch.distributed as dist
 
     def all_reduce(t):
-        dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+        if accumulate_in_fp32 and t.dtype in (torch.bfloat16, torch.float16):
+            wide = t.float()
+            dist.all_reduce(wide, op=dist.ReduceOp.SUM, group=group)
+            t.copy_(wide)
+        else:
+            dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
 
     return all_reduce

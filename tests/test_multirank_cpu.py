@@ -118,3 +118,32 @@ def test_shard_ranges_cover_the_hidden_dimension():
         parallel.shard_range(20, 0, 2)
     with pytest.raises(ValueError):
         parallel.shard_range(16, 0, 3)
+
+
+# ---- the all-reduce of 16-bit partial tensors accumulates in fp32 and rounds once ---------------------------------
+def _bf16_sum_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    from paper_2405_03133_b200 import parallel
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ulp = 2.0 ** -7                                   # spacing of bf16 numbers in [1, 2)
+    # rank 0 contributes 1, the other two 0.3 ulp each: a running bf16 sum stays at 1 (each addend is below half
+    # an ulp), the fp32 sum is 1 + 0.6 ulp and rounds to 1 + 1 ulp
+    mine = 1.0 if rank == 0 else 0.3 * ulp
+    t = torch.full((4,), mine, dtype=torch.bfloat16)
+    parallel.torch_all_reduce()(t)
+    out[rank] = t.float().tolist()
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_all_reduce_of_bf16_partials_rounds_once():
+    world = 3
+    port = 33000 + os.getpid() % 2000
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_bf16_sum_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    for r in range(world):
+        assert res[r] == [1.0 + 2.0 ** -7] * 4
