@@ -46,7 +46,9 @@ typedef enum {
   LORY_ERR_ARCH = -5,           /* current device is not compute capability 10.x               */
   LORY_ERR_CUDA = -6,           /* a CUDA runtime/driver call failed (see lory_last_cuda_error)*/
   LORY_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait expired (lory_check_status)      */
-  LORY_ERR_TOO_LARGE = -8       /* problem exceeds the fixed scratch of lory_route_noalloc     */
+  LORY_ERR_TOO_LARGE = -8,      /* problem exceeds the fixed scratch of lory_route_noalloc     */
+  LORY_ERR_DEBUG_BOUNDS = -9    /* debug build: a tile coordinate, shared-memory stage or TMEM
+                                   column range was out of bounds (lory_check_status)          */
 } lory_status;
 
 typedef enum { LORY_FP32 = 0, LORY_BF16 = 1 } lory_dtype;
@@ -221,8 +223,9 @@ int lory_moe_step_host_wait(int slot);
 
 /*
  * Reads the device status word kept in the workspace (synchronises the stream).
- * Returns LORY_OK, or LORY_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up,
- * in which case the outputs of that call are undefined.
+ * Returns LORY_OK, or LORY_ERR_DEBUG_BOUNDS if a bounds check of the debug build fired, or
+ * LORY_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up; in both cases the outputs of that
+ * call are undefined.
  */
 int lory_check_status(const lory_dims* dims, void* workspace, size_t workspace_bytes,
                       void* cuda_stream);
@@ -269,6 +272,25 @@ int lory_route_noalloc(const lory_dims* dims, const void* x, const void* w_r, fl
  * status word first.  The kernels of the layer use the same bounded wait with a much larger limit.
  */
 int lory_selftest_bounded_wait(const lory_dims* dims, void* workspace, size_t workspace_bytes,
+                               void* cuda_stream);
+
+/*
+ * Debug build.  The library can be built a second time with -DLORY_DEBUG
+ * (python -m paper_2405_03133_b200.build --debug -> liblory_debug.so; same ABI).  Its tensor-core kernels
+ * check, before use, every tile coordinate they hand to the TMA engine (range against the padded problem
+ * extents, 16-byte alignment of the innermost coordinate), every shared-memory stage and staging buffer
+ * against the CTA's allocation, and every TMEM column range against the allocated columns.  A violated
+ * bound sets a bit in the status word and the access is skipped (stores, MMAs) or redirected to coordinate
+ * zero (loads) rather than issued; lory_check_status then returns LORY_ERR_DEBUG_BOUNDS.  This is the
+ * tool for hunting an out-of-range index without a memory checker; it costs a few per cent of run time.
+ *   lory_debug_build()            1 in the debug build, 0 in the release build.
+ *   lory_selftest_debug_bounds()  makes the three kinds of check fire on purpose, on made-up values and
+ *                                 without any access: in the debug build a following lory_check_status
+ *                                 returns LORY_ERR_DEBUG_BOUNDS, in the release build LORY_OK (the checks
+ *                                 are compiled out).  Clears the status word first.
+ */
+int lory_debug_build(void);
+int lory_selftest_debug_bounds(const lory_dims* dims, void* workspace, size_t workspace_bytes,
                                void* cuda_stream);
 
 /*

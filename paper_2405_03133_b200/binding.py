@@ -18,7 +18,8 @@ LORY_FLAG_FIRST_SEGMENT_GRAD = 8
 LORY_FLAG_ACCUMULATE_GRADS = 16
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liblory.so")
+# LORY_LIBRARY selects another build of the same ABI, e.g. the bounds-checking liblory_debug.so
+LIB_PATH = os.environ.get("LORY_LIBRARY") or os.path.join(_HERE, "liblory.so")
 
 
 class LoryError(RuntimeError):
@@ -59,6 +60,8 @@ _SIGNATURES = {
     "lory_route_noalloc": (ctypes.c_int, [_DP] + [_vp] * 5),
     "lory_expert_utilization": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int, _vp, _vp]),
     "lory_selftest_bounded_wait": (ctypes.c_int, [_DP, _vp, _sz, _vp]),
+    "lory_debug_build": (ctypes.c_int, []),
+    "lory_selftest_debug_bounds": (ctypes.c_int, [_DP, _vp, _sz, _vp]),
     "lory_probe_l2_ring": (ctypes.c_int, [_vp, _sz, _sz] + [ctypes.c_int] * 5 + [ctypes.POINTER(ctypes.c_float), _vp]),
     "lory_profile_enable": (ctypes.c_int, [ctypes.c_int]),
     "lory_profile_read": (ctypes.c_int, [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)]),
@@ -247,3 +250,13 @@ def lory_probe_l2_ring(buf, slot_bytes, slots, lag, iters, mode=3, shift=0, stre
     _check(load().lory_probe_l2_ring(_ptr(buf), _nbytes(buf), int(slot_bytes), int(slots), int(lag), int(iters),
                                      int(mode), int(shift), ctypes.byref(ms), _stream(stream)))
     return ms.value
+
+
+def lory_debug_build():
+    """1 if the loaded library is the bounds-checking debug build, else 0."""
+    return load().lory_debug_build()
+
+
+def lory_selftest_debug_bounds(dims, workspace, stream=None):
+    """Makes the debug build's bounds checks fire on made-up values; lory_check_status then reports them."""
+    _check(load().lory_selftest_debug_bounds(ctypes.byref(dims), _ptr(workspace), _nbytes(workspace), _stream(stream)))

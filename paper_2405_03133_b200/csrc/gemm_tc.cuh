@@ -210,10 +210,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         const int rest = tile / p.m_tiles;
         const int n_tile = rest % p.n_tiles;
         const int g = rest / p.n_tiles;
-        const int m0 = m_tile * (128 * CTAS) + 128 * rank, n0 = n_tile * TILE_N;
-        const int gc = g;
+        int m0 = m_tile * (128 * CTAS) + 128 * rank, n0 = n_tile * TILE_N;
+        int gc = g;
         const int nkb = (p.K + 63) / 64;
         const int total = (MODE == MODE_DUALK) ? 2 * nkb : nkb;
+        // debug build: the tile's coordinates against the padded problem extents (a violated bound is recorded
+        // and the tile is loaded from coordinate zero instead, so that every barrier still completes)
+        if (!dbg::check(dbg::inner_ok(m0, p.m_tiles * 128 * CTAS) && dbg::inner_ok(n0, p.n_tiles * TILE_N) &&
+                            dbg::coord_ok(gc, p.groups),
+                        p.status)) {
+          m0 = 128 * rank;
+          n0 = 0;
+          gc = 0;
+        }
         for (int i = 0; i < total; ++i, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
@@ -224,11 +233,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           }
           const bool second = (MODE == MODE_DUALK) && (i >= nkb);
           const int kb = second ? i - nkb : i;
-          const int kc = kb * 64;
+          const int kc = dbg::check(dbg::inner_ok(kb * 64, nkb * 64), p.status) ? kb * 64 : 0;
           const CUtensorMap* ta = second ? &tmA1 : &tmA0;
           const CUtensorMap* tb = second ? &tmB1 : &tmB0;
           uint8_t* sA = smem + (size_t)s * Tile::STAGE_BYTES;
           uint8_t* sB = sA + Tile::A_BYTES;
+          // a stage outside the shared-memory allocation is never written: the consumer's bounded wait reports it
+          if (!dbg::check(dbg::smem_ok(sA, Tile::STAGE_BYTES), p.status)) continue;
           if (!PAIR) ptx::mbar_expect_tx(&full_bar[s], Tile::STAGE_BYTES);
           else if (rank == 0) ptx::mbar_expect_tx(&full_bar[s], 2 * Tile::STAGE_BYTES);  // both CTAs' bytes land here
           issued |= 1u << s;
@@ -301,6 +312,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         }
         ptx::tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + acc * BN;
+        const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d, tmem_base, 2 * BN, BN), p.status);
         for (int i = 0; i < total; ++i, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
@@ -317,6 +329,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                                         : ptx::make_smem_desc(a_addr + k16 * 32, 16, 1024);
             const uint64_t bdesc = B_MN ? ptx::make_smem_desc(b_addr + k16 * 2048, 8192, 1024)
                                         : ptx::make_smem_desc(b_addr + k16 * 32, 16, 1024);
+            if (!acc_ok) continue;  // debug build: an accumulator outside the TMEM allocation is never written
             if (PAIR) ptx::umma_bf16_pair(tmem_d, adesc, bdesc, idesc, (i > 0 || k16 > 0) ? 1u : 0u);
             else ptx::umma_bf16(tmem_d, adesc, bdesc, idesc, (i > 0 || k16 > 0) ? 1u : 0u);
           }
@@ -343,6 +356,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     WarpStager wsg;  // per-warp staging (all other epilogues)
     wsg.buf = os.buf + q * 8192;
     wsg.n = 0;
+    const bool staging_ok = dbg::check(dbg::smem_ok(os.buf, 2 * Tile::OUT_BYTES + Tile::IN_BYTES), p.status);
     uint32_t tile_iter = 0;
     for (int tile = wid; tile < num_tiles; tile += wstride, ++tile_iter) {
       const int m_tile = tile % p.m_tiles;
@@ -359,6 +373,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       __syncwarp();  // every lane polls by itself; the warp-wide tcgen05 instructions below need it whole again
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+      // debug build: this tile's output coordinates and accumulator columns; a tile that fails is drained
+      // (its accumulator handed back) without reading TMEM or storing anything
+      if (!dbg::check(staging_ok && dbg::inner_ok(n0, p.n_tiles * TILE_N) &&
+                          dbg::coord_ok(m0, p.m_tiles * 128 * CTAS) && dbg::coord_ok(g, p.groups) &&
+                          dbg::tmem_ok(taddr, tmem_base, 2 * BN, BN),
+                      p.status)) {
+        ptx::tc_fence_before_sync();
+        arrive_tmem_empty(&tmem_empty_bar[acc]);
+        continue;
+      }
 
       if (EPI == EPI_BF16 || EPI == EPI_BF16_ROWADD || EPI == EPI_BF16_RESADD) {
         // software pipeline: the TMEM load of the next 64-column group is in flight while the

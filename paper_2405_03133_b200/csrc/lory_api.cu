@@ -349,6 +349,7 @@ const char* lory_status_string(int status) {
     case LORY_ERR_CUDA: return "LORY_ERR_CUDA: a CUDA call failed";
     case LORY_ERR_DEVICE_TIMEOUT: return "LORY_ERR_DEVICE_TIMEOUT: a bounded device-side wait expired";
     case LORY_ERR_TOO_LARGE: return "LORY_ERR_TOO_LARGE: problem exceeds the fixed scratch array of lory_route_noalloc";
+    case LORY_ERR_DEBUG_BOUNDS: return "LORY_ERR_DEBUG_BOUNDS: a bounds check of the debug build fired";
     default: return "unknown lory_status";
   }
 }
@@ -793,7 +794,23 @@ int lory_check_status(const lory_dims* dims, void* workspace, size_t workspace_b
   cudaStream_t st = (cudaStream_t)cuda_stream;
   LORY_CUDA_OK(cudaMemcpyAsync(&word, (char*)workspace + Lo.status, 4, cudaMemcpyDeviceToHost, st));
   LORY_CUDA_OK(cudaStreamSynchronize(st));
+  if (word & STATUS_DEBUG_BOUNDS) return LORY_ERR_DEBUG_BOUNDS;
   return word == 0 ? LORY_OK : LORY_ERR_DEVICE_TIMEOUT;
+}
+
+int lory_debug_build(void) { return dbg::kOn ? 1 : 0; }
+
+int lory_selftest_debug_bounds(const lory_dims* dims, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int s = check_dims(dims);
+  if (s != LORY_OK) return s;
+  Layout Lo = make_layout(*dims);
+  s = check_ws(workspace, workspace_bytes, Lo.fwd_end);
+  if (s != LORY_OK) return s;
+  s = check_device();
+  if (s != LORY_OK) return s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  LORY_CUDA_OK(cudaMemsetAsync((char*)workspace + Lo.status, 0, 256, st));
+  return tc_debug_bounds_selftest((uint32_t*)((char*)workspace + Lo.status), st);
 }
 
 }  // extern "C"

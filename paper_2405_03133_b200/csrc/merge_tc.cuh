@@ -89,6 +89,14 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
     c0 = (rem >> 6) * 256;
   };
 
+  // debug build: a decoded tile against the padded tile grid of its matrix
+  auto tile_ok = [&](int k, int r, int c0) {
+    if (!dbg::kOn) return true;
+    if (k < 0 || k > 2) return false;
+    const int tiles_k = p.tile_end[k] - (k ? p.tile_end[k - 1] : 0);
+    return dbg::coord_ok(r, tiles_k / p.ctiles[k]) && dbg::inner_ok(c0, p.ctiles[k] * 256);
+  };
+
   if (warp == 0) {
     if (lane == 0) {
       ptx::mbar_expect_tx(&w_bar, (uint32_t)p.s_tiles * 32768u);
@@ -108,6 +116,10 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
         int k, r, c0;
         decode(tile, k, r, c0);
+        // debug build: matrix index, row and first column of the tile against the padded tile grid
+        if (!dbg::check(tile_ok(k, r, c0), p.status)) {
+          k = 0; r = 0; c0 = 0;
+        }
         const int s = it % STAGES;
         const uint32_t ph = (it / STAGES) & 1;
         if (!ptx::mbar_wait(&empty_bar[s], ph ^ 1, &abort_flag)) {
@@ -115,6 +127,7 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
           abort_flag = 1;
         }
         uint8_t* sB = s_stage + (size_t)s * p.stage_bytes;
+        if (!dbg::check(dbg::smem_ok(sB, (uint32_t)p.stage_bytes), p.status)) continue;
         ptx::mbar_expect_tx(&full_bar[s], (uint32_t)p.stage_bytes);
         issued |= 1u << s;
         last_parity = (last_parity & ~(1u << s)) | (ph << s);
@@ -154,7 +167,8 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
           ptx::tc_fence_after_sync();
           const uint32_t tmem_d = tmem_base + acc * 256;
           const uint32_t a_hi = wbase + st * 32768, a_lo = a_hi + 16384;
-          for (int kk = 0; kk < ksteps; ++kk) {
+          const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d, tmem_base, 512, 256) && st < 2, p.status);
+          for (int kk = 0; kk < ksteps && acc_ok; ++kk) {
             const uint64_t bdesc = ptx::make_smem_desc(bbase + kk * 2048, lbo, 1024);
             ptx::umma_bf16(tmem_d, ptx::make_smem_desc(a_hi + kk * 32, 16, 1024), bdesc, idesc, kk > 0 ? 1u : 0u);
             ptx::umma_bf16(tmem_d, ptx::make_smem_desc(a_lo + kk * 32, 16, 1024), bdesc, idesc, 1u);
@@ -186,6 +200,16 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
         __syncwarp();  // every lane polls by itself; the warp-wide tcgen05 instructions below need it whole again
         ptx::tc_fence_after_sync();
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
+        // debug build: accumulator columns, staging buffer and output coordinates of this warp's stores; a tile
+        // that fails is drained without reading TMEM or storing
+        if (!dbg::check(dbg::tmem_ok(taddr + c_begin * 64, tmem_base, 512, (c_end - c_begin) * 64) &&
+                            dbg::smem_ok(wsg.buf, 8192) && tile_ok(k, r, c0) &&
+                            dbg::coord_ok(st * 128 + seg0, p.s_tiles * 128),
+                        p.status)) {
+          ptx::tc_fence_before_sync();
+          ptx::mbar_arrive(&tmem_empty_bar[acc]);
+          continue;
+        }
         uint32_t rr[64];
         ptx::tmem_ld_32x64(taddr + c_begin * 64, rr);
 #pragma unroll 1

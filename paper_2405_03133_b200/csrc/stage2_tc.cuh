@@ -74,6 +74,14 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
     c0 = (local - r * p.ctiles[k]) * 128;
   };
 
+  // debug build: a decoded tile against the padded tile grid of its matrix
+  auto tile_ok = [&](int k, int r, int c0) {
+    if (!dbg::kOn) return true;
+    if (k < 0 || k > 2) return false;
+    const int tiles_k = p.tile_end[k] - (k ? p.tile_end[k - 1] : 0);
+    return dbg::coord_ok(r, tiles_k / p.ctiles[k]) && dbg::inner_ok(c0, p.ctiles[k] * 128);
+  };
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < 8; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
@@ -115,6 +123,9 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
         int k, r, c0;
         decode(tile, k, r, c0);
+        if (!dbg::check(tile_ok(k, r, c0), p.status)) {
+          k = 0; r = 0; c0 = 0;
+        }
         for (int st = 0; st < p.s_tiles; ++st, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
@@ -124,6 +135,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           }
           uint8_t* sD = s_stage + (size_t)s * p.stage_bytes;
           uint8_t* sT = sD + 2 * p.cb_stride;
+          if (!dbg::check(dbg::smem_ok(sD, (uint32_t)p.stage_bytes) && dbg::coord_ok(st, 2), p.status)) continue;
           ptx::mbar_expect_tx(&full_bar[s], tx);
           issued |= 1u << s;
           last_parity = (last_parity & ~(1u << s)) | (ph << s);
@@ -155,6 +167,10 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           abort_flag = 1;
         }
         const uint32_t tmem_d1 = tmem_base + acc * 128;
+        // debug build: both accumulators (the per-tile one and the resident dw one) inside the 512 columns
+        const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d1, tmem_base, 512, 128) &&
+                                           dbg::tmem_ok(tmem_d2, tmem_base, 512, (uint32_t)(p.s_tiles * p.Epad16)),
+                                       p.status);
         for (int st = 0; st < p.s_tiles; ++st, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
@@ -170,7 +186,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           const int ksteps = (rows + 15) / 16;
           // rows 0..63: w_hi^T [e, s] . dWbar [s, p]; rows 64..127: w_lo^T . dWbar (the A operand's second
           // 64-row group lies 16 KB after the first: that is the lo tile)
-          for (int kk = 0; kk < ksteps; ++kk) {
+          for (int kk = 0; kk < ksteps && acc_ok; ++kk) {
             ptx::umma_bf16(tmem_d1, ptx::make_smem_desc(whi + kk * 2048, 16384, 1024),
                            ptx::make_smem_desc(dbase + kk * 2048, (uint32_t)p.cb_stride, 1024), idesc1,
                            (st > 0 || kk > 0) ? 1u : 0u);
@@ -183,6 +199,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           for (int j = 0; j < 2; ++j) {
 #pragma unroll
             for (int k16 = 0; k16 < 4; ++k16) {
+              if (!acc_ok) continue;
               const uint64_t adesc = ptx::make_smem_desc(dbase + j * p.cb_stride + k16 * 32, 16, 1024);
               const uint64_t bdesc = ptx::make_smem_desc(tbase + j * p.Epad16 * 128 + k16 * 32, 16, 1024);
               ptx::umma_bf16(tmem_d2s, adesc, bdesc, idesc2, (tcount > 0 || j > 0 || k16 > 0) ? 1u : 0u);
@@ -225,7 +242,13 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
       __syncwarp();  // every lane polls by itself; the warp-wide tcgen05 instructions below need it whole again
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 128;
-      if (!has_rows) {
+      // debug build: a tile whose coordinates, accumulator columns or staging buffers are out of range is drained
+      // (every term is the same for the two warps of a couple, which meet at a named barrier below)
+      const bool tile_fine = dbg::check(tile_ok(k, row, c0) && dbg::tmem_ok(taddr, tmem_base, 512, 128) &&
+                                            dbg::smem_ok(wsg.buf, 8192) &&
+                                            dbg::smem_ok(s_xch + pair * 2 * p.xch_bytes, 2u * (uint32_t)p.xch_bytes),
+                                        p.status);
+      if (!has_rows || !tile_fine) {
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(&tmem_empty_bar[acc]);
         continue;

@@ -543,6 +543,23 @@ __global__ void bounded_wait_selftest_kernel(uint32_t* status, uint32_t limit) {
   }
 }
 
+// The three predicates of the debug build on values that must fail each of them; nothing is accessed.
+__global__ void debug_bounds_selftest_kernel(uint32_t* status) {
+  extern __shared__ uint8_t dyn[];
+  // (a) a tile coordinate: negative, beyond the extent, or off the 16-byte grid
+  dbg::check(dbg::coord_ok(-1, 8) || dbg::coord_ok(8, 8) || dbg::inner_ok(4, 64), status);
+  // (b) a shared-memory stage that ends one byte after the 1024 bytes this launch was given
+  dbg::check(dbg::smem_ok(dyn + 1, 1024), status);
+  // (c) a TMEM column range: 64 columns starting at column 480 of a 512-column allocation
+  dbg::check(dbg::tmem_ok(480u, 0u, 512u, 64u), status);
+}
+
+int tc_debug_bounds_selftest(uint32_t* status_word, cudaStream_t st) {
+  debug_bounds_selftest_kernel<<<1, 1, 1024, st>>>(status_word);
+  LORY_AFTER_LAUNCH();
+  return LORY_OK;
+}
+
 int tc_bounded_wait_selftest(uint32_t* status_word, cudaStream_t st) {
   bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(status_word, 10000u);
   LORY_AFTER_LAUNCH();

@@ -32,6 +32,10 @@ int tc_ffn_backward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* 
 int tc_ffn_backward_dx(const lory_dims& D, const Layout& Lo, char* ws, const float* dh_bar, bf16* dx,
                        cudaStream_t st);
 
+// Evaluates the debug build's three kinds of bounds check on made-up out-of-range values (no access is made):
+// raises STATUS_DEBUG_BOUNDS in a debug build, nothing in a release build.
+int tc_debug_bounds_selftest(uint32_t* status_word, cudaStream_t st);
+
 // Launches a one-thread kernel whose bounded mbarrier wait must expire and raise the status word.
 int tc_bounded_wait_selftest(uint32_t* status_word, cudaStream_t st);
 

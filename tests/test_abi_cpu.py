@@ -38,9 +38,24 @@ def test_exports_every_declared_symbol(lib):
     assert set(names) == set(lory.binding.exported_symbols())
 
 
+def test_debug_build_exports_the_same_symbols():
+    """The bounds-checking build (-DLORY_DEBUG) has the same ABI and says what it is."""
+    if shutil.which("nvcc") is None and not os.path.exists(lory_build.LIB_DEBUG):
+        pytest.skip("liblory_debug.so not built and nvcc not available")
+    dbg = ctypes.CDLL(lory_build.build(debug=True))
+    for n in declared_functions():
+        assert hasattr(dbg, n), f"{n} missing from the debug build"
+    dbg.lory_debug_build.restype = ctypes.c_int
+    assert dbg.lory_debug_build() == 1
+
+
+def test_release_build_is_not_the_debug_build(lib):
+    assert lory.binding.lory_debug_build() == 0
+
+
 def test_status_strings(lib):
     assert lory.lory_status_string(0) == "LORY_OK"
-    for code in range(-8, 0):
+    for code in range(-9, 0):
         assert lory.lory_status_string(code).startswith("LORY_ERR_")
     assert "unknown" in lory.lory_status_string(-99)
 
