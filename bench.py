@@ -271,6 +271,63 @@ def workload_config(wl):
             "tokens_per_step": wl.tokens, "l2": "working set (merged weights, activations: several GB) exceeds L2; no flush"}
 
 
+def run_decode(args, wl):
+    """Prompt-only routing at inference (Section 3.1): one prefill over the prompt fixes a merged FFN per sequence;
+    every later call applies it to n new tokens per sequence.  A call has to read each sequence's merged weights
+    once (B * 3 * d * f * 2 bytes) whatever n is, so it is bound by HBM: reported are the device time per call
+    (CUDA events over a run of back-to-back calls), tokens/s, the merged-weight bytes over that time against the
+    measured copy bandwidth, and the host time the call itself takes (the floor of a latency-bound decode loop)."""
+    import torch
+    import paper_2405_03133_b200 as lory
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4321)
+
+    def normal(shape, std):
+        return (torch.randn(shape, generator=gen, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
+
+    peaks = load_peaks()
+    w_r, W1 = normal((wl.E, wl.d), 0.02), normal((wl.E, wl.f, wl.d), 0.02)
+    W2, W3 = normal((wl.E, wl.d, wl.f), 0.02), normal((wl.E, wl.f, wl.d), 0.02)
+    prompt = normal((wl.B, wl.L, wl.d), 1.0)
+    pdims = lory.make_dims(wl.B, wl.L, wl.L, wl.d, wl.f, wl.E, "bf16")
+    fwd_b, _ = lory.lory_moe_workspace_bytes(pdims)
+    ws = torch.empty(fwd_b, dtype=torch.uint8, device=dev)
+    y = torch.empty_like(prompt)
+    rw = torch.empty((wl.B, wl.E), dtype=torch.float32, device=dev)
+    lory.lory_moe_forward(pdims, prompt, w_r, W1, W2, W3, y, rw, None, ws)
+    lory.lory_check_status(pdims, ws)
+    merged_bytes = wl.B * 3 * wl.d * wl.f * 2
+    rows = []
+    for n in (1, 4, 16, 64):
+        ddims = lory.make_dims(wl.B, n, n, wl.d, wl.f, wl.E, "bf16", lory.LORY_FLAG_REUSE_MERGED)
+        x_new = normal((wl.B, n, wl.d), 1.0)
+        y_new = torch.empty_like(x_new)
+        for _ in range(max(args.warmup, 3)):
+            lory.lory_moe_ffn(ddims, x_new, None, W1, W2, W3, y_new, ws)
+        torch.cuda.synchronize()
+        calls = 200
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        ev0.record()
+        for _ in range(calls):
+            lory.lory_moe_ffn(ddims, x_new, None, W1, W2, W3, y_new, ws)
+        ev1.record()
+        host_us = (time.perf_counter() - t0) / calls * 1e6
+        torch.cuda.synchronize()
+        dev_us = ev0.elapsed_time(ev1) / calls * 1e3
+        lory.lory_check_status(ddims, ws)
+        rows.append({"new_tokens_per_sequence": n, "device_us_per_call": dev_us, "host_us_per_call": host_us,
+                     "tokens_per_s": wl.B * n / (dev_us * 1e-6), "launches_per_call": lory.lory_last_launch_count(),
+                     "merged_weight_gbs": merged_bytes / (dev_us * 1e-6) / 1e9,
+                     "frac_of_hbm_peak": merged_bytes / (dev_us * 1e-6) / 1e9 / peaks["hbm_gbs"]})
+    print(json.dumps({"metric": "Lory prompt-routed decode (cached merged FFN), tokens/s", "unit": UNIT,
+                      "config": {"workload": f"{wl.name}: B={wl.B} prompt={wl.L} d_model={wl.d} d_ff={wl.f} E={wl.E} bf16",
+                                 "merged_weight_bytes_per_call": merged_bytes}, "dtype": "bf16", "data": "synthetic",
+                      "hbm_peak_gbs": peaks["hbm_gbs"], "calls": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -282,6 +339,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sustained", action="store_true", help="skip the second timed region of >= 1 s")
+    ap.add_argument("--decode", action="store_true",
+                    help="measure the inference path instead: prefill with prompt-only routing, then decode calls")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -291,6 +350,9 @@ def main():
         wl = wl.with_(B=args.batch, name=f"{wl.name}_B{args.batch}")
     if args.impl == "reference":
         run_reference(args, wl)
+        return
+    if args.decode:
+        run_decode(args, wl)
         return
 
     import torch

@@ -33,6 +33,7 @@ struct Stage2Params {
   int S, E, Epad16, s_tiles;  // S: segments of this launch (at most 256); s_tiles = ceil(S / 128)
   int seg_base, S_total;      // first segment of this launch; all segments (row count of a dw slab)
   int ctiles[3];    // 128-column tiles per row
+  uint32_t cmagic[3];  // ceil(2^32 / ctiles), 0 for ctiles == 1: n / ctiles == __umulhi(n, cmagic) for every tile index n
   int tile_end[3];  // exclusive prefix sums of (rows rounded up to 64) * ctiles
   int cb_stride;    // bytes between the two 64-column blocks of a dWbar tile in shared memory (= segments per box * 128)
   int dup;          // E <= 32: w_hi and w_lo are both the combined [hi (32) | lo (32)] table
@@ -70,7 +71,8 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   auto decode = [&](int tile, int& k, int& r, int& c0) {
     k = tile < p.tile_end[0] ? 0 : (tile < p.tile_end[1] ? 1 : 2);
     const int local = tile - (k == 0 ? 0 : p.tile_end[k - 1]);
-    r = local / p.ctiles[k];
+    // local / ctiles[k] without the division (a single tile per row has no 32-bit reciprocal: magic 0)
+    r = p.cmagic[k] ? (int)__umulhi((uint32_t)local, p.cmagic[k]) : local;
     c0 = (local - r * p.ctiles[k]) * 128;
   };
 
@@ -118,7 +120,9 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
         ptx::tma_load_3d(s_w + st * 32768, &maps.w_hi, &w_bar, 0, p.seg_base + st * 128, 0);
         ptx::tma_load_3d(s_w + st * 32768 + 16384, &maps.w_lo, &w_bar, 0, p.seg_base + st * 128, 0);
       }
-      uint32_t it = 0, issued = 0, last_parity = 0;
+      uint32_t issued = 0, last_parity = 0;
+      int s = 0;          // position in the stage ring and its phase, advanced by hand: a division per tile on
+      uint32_t ph = 0;    // this one thread is time the whole pipeline waits for
       const uint32_t tx = (uint32_t)p.tx_bytes;
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
         int k, r, c0;
@@ -126,9 +130,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
         if (!dbg::check(tile_ok(k, r, c0), p.status)) {
           k = 0; r = 0; c0 = 0;
         }
-        for (int st = 0; st < p.s_tiles; ++st, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+        for (int st = 0; st < p.s_tiles; ++st, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0)) {
           if (!ptx::mbar_wait(&empty_bar[s], ph ^ 1, &abort_flag)) {
             atomicOr(p.status, STATUS_TIMEOUT_TMA);
             abort_flag = 1;
@@ -159,7 +161,16 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
         abort_flag = 1;
       }
       const uint32_t wbase = ptx::smem_u32(s_w);
-      uint32_t it = 0, tcount = 0;
+      // Shared-memory descriptors differ only in their 14-bit address field (16-byte units): the constant part is
+      // built once and the address added per instruction, which keeps this one thread's work per tile small.
+      const uint64_t d1a = ptx::make_smem_desc(0, 16384, 1024);                    // w tile, lo 16 KB behind hi
+      const uint64_t d1b = ptx::make_smem_desc(0, (uint32_t)p.cb_stride, 1024);    // dWbar tile as [segment, column]
+      const uint64_t d2ab = ptx::make_smem_desc(0, 16, 1024);                      // K-major tiles of the second product
+      const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4, cb16 = (uint32_t)p.cb_stride >> 4;
+      const uint32_t t16 = (uint32_t)(p.Epad16 * 128) >> 4;
+      const uint32_t stage0_16 = ptx::smem_u32(s_stage) >> 4, w16 = wbase >> 4;
+      int s = 0;
+      uint32_t ph = 0, tcount = 0;
       for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tcount) {
         const uint32_t acc = tcount & 1;
         if (!ptx::mbar_wait(&tmem_empty_bar[acc], ((tcount >> 1) & 1) ^ 1, &abort_flag)) {
@@ -171,24 +182,21 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
         const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d1, tmem_base, 512, 128) &&
                                            dbg::tmem_ok(tmem_d2, tmem_base, 512, (uint32_t)(p.s_tiles * p.Epad16)),
                                        p.status);
-        for (int st = 0; st < p.s_tiles; ++st, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+        for (int st = 0; st < p.s_tiles; ++st, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0)) {
           if (!ptx::mbar_wait(&full_bar[s], ph, &abort_flag)) {
             atomicOr(p.status, STATUS_TIMEOUT_MMA);
             abort_flag = 1;
           }
           ptx::tc_fence_after_sync();
-          const uint32_t dbase = ptx::smem_u32(s_stage + (size_t)s * p.stage_bytes);
-          const uint32_t tbase = dbase + 2 * p.cb_stride;
-          const uint32_t whi = wbase + st * 32768;
+          const uint32_t d16 = stage0_16 + (uint32_t)s * stage16;   // this stage's dWbar tile, 16-byte units
+          const uint32_t tb16 = d16 + 2 * cb16;                     // its expert tile
+          const uint32_t whi16 = w16 + (uint32_t)st * (32768u >> 4);
           const int rows = min(128, p.S - st * 128);
           const int ksteps = (rows + 15) / 16;
           // rows 0..63: w_hi^T [e, s] . dWbar [s, p]; rows 64..127: w_lo^T . dWbar (the A operand's second
           // 64-row group lies 16 KB after the first: that is the lo tile)
           for (int kk = 0; kk < ksteps && acc_ok; ++kk) {
-            ptx::umma_bf16(tmem_d1, ptx::make_smem_desc(whi + kk * 2048, 16384, 1024),
-                           ptx::make_smem_desc(dbase + kk * 2048, (uint32_t)p.cb_stride, 1024), idesc1,
+            ptx::umma_bf16(tmem_d1, d1a | (uint64_t)(whi16 + kk * 128), d1b | (uint64_t)(d16 + kk * 128), idesc1,
                            (st > 0 || kk > 0) ? 1u : 0u);
           }
           // dw [s, e] += dWbar [s, p] . W^T [p, e]   (one accumulator per group of 128 segments; with fewer than
@@ -200,8 +208,8 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
 #pragma unroll
             for (int k16 = 0; k16 < 4; ++k16) {
               if (!acc_ok) continue;
-              const uint64_t adesc = ptx::make_smem_desc(dbase + j * p.cb_stride + k16 * 32, 16, 1024);
-              const uint64_t bdesc = ptx::make_smem_desc(tbase + j * p.Epad16 * 128 + k16 * 32, 16, 1024);
+              const uint64_t adesc = d2ab | (uint64_t)(d16 + j * cb16 + k16 * 2);
+              const uint64_t bdesc = d2ab | (uint64_t)(tb16 + j * t16 + k16 * 2);
               ptx::umma_bf16(tmem_d2s, adesc, bdesc, idesc2, (tcount > 0 || j > 0 || k16 > 0) ? 1u : 0u);
             }
           }

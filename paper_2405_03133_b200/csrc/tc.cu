@@ -314,6 +314,9 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const bf16* const 
   p.S = S_launch; p.S_total = S; p.E = E; p.Epad16 = e_pad16(D); p.s_tiles = (S_launch + 127) / 128;
   p.dw_partial = q.dw_partial; p.status = q.status;
   stage2_tiles(D, p.ctiles, p.tile_end);
+  for (int k = 0; k < 3; ++k)
+    p.cmagic[k] = p.ctiles[k] == 1 ? 0u : (uint32_t)(((1ull << 32) + p.ctiles[k] - 1) / p.ctiles[k]);
+  if ((uint64_t)p.tile_end[2] * 64 >= (1ull << 32)) return LORY_ERR_SHAPE;  // keeps the reciprocal division exact
   // A box of fewer than 128 segments when S < 128: TMA would otherwise zero-fill the missing rows piece by piece.
   // A multiple of 16, so that the K steps of the first product stay inside the box (rows S.. of it are zero-filled).
   const uint32_t seg_box = S >= 128 ? 128u : (uint32_t)((S + 15) / 16 * 16);
