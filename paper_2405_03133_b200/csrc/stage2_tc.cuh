@@ -58,8 +58,9 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   uint8_t* s_stage = s_xch + 4 * p.xch_bytes;
   __shared__ __align__(8) uint64_t full_bar[8];
   __shared__ __align__(8) uint64_t empty_bar[8];
-  __shared__ __align__(8) uint64_t tmem_full_bar[2];
-  __shared__ __align__(8) uint64_t tmem_empty_bar[2];
+  constexpr int NACC = 2;  // per-tile accumulators in flight (three were measured: no faster), the dw accumulator behind them
+  __shared__ __align__(8) uint64_t tmem_full_bar[NACC];
+  __shared__ __align__(8) uint64_t tmem_empty_bar[NACC];
   __shared__ __align__(8) uint64_t w_bar, d2_bar;
   __shared__ uint32_t tmem_base_smem;
   __shared__ volatile uint32_t abort_flag;
@@ -89,7 +90,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
       ptx::mbar_init(&full_bar[s], 1);
       ptx::mbar_init(&empty_bar[s], 1);
     }
-    for (int a = 0; a < 2; ++a) {
+    for (int a = 0; a < NACC; ++a) {
       ptx::mbar_init(&tmem_full_bar[a], 1);
       ptx::mbar_init(&tmem_empty_bar[a], 128);
     }
@@ -110,7 +111,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_smem;
-  const uint32_t tmem_d2 = tmem_base + 256;
+  const uint32_t tmem_d2 = tmem_base + NACC * 128;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -171,9 +172,10 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
       const uint32_t stage0_16 = ptx::smem_u32(s_stage) >> 4, w16 = wbase >> 4;
       int s = 0;
       uint32_t ph = 0, tcount = 0;
-      for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tcount) {
-        const uint32_t acc = tcount & 1;
-        if (!ptx::mbar_wait(&tmem_empty_bar[acc], ((tcount >> 1) & 1) ^ 1, &abort_flag)) {
+      uint32_t acc = 0, acc_ph = 0;   // accumulator ring position and phase
+      for (int tile = blockIdx.x; tile < num_tiles;
+           tile += gridDim.x, ++tcount, acc = (acc + 1 == NACC ? 0 : acc + 1), acc_ph ^= (acc == 0)) {
+        if (!ptx::mbar_wait(&tmem_empty_bar[acc], acc_ph ^ 1, &abort_flag)) {
           atomicOr(p.status, STATUS_TIMEOUT_MMA);
           abort_flag = 1;
         }
@@ -239,11 +241,12 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
     const int xlane = p.xch_bytes >> 5, xmask = (xlane >> 4) - 1;
     uint8_t* xch = s_xch + pair * 2 * p.xch_bytes + lane * xlane;
     uint32_t it = 0;
-    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+    uint32_t acc = 0, acc_ph = 0;   // accumulator ring position and phase
+    for (int tile = blockIdx.x; tile < num_tiles;
+         tile += gridDim.x, ++it, acc = (acc + 1 == NACC ? 0 : acc + 1), acc_ph ^= (acc == 0)) {
       int k, row, c0;
       decode(tile, k, row, c0);
-      const uint32_t acc = it & 1;
-      if (!ptx::mbar_wait(&tmem_full_bar[acc], (it >> 1) & 1, &abort_flag)) {
+      if (!ptx::mbar_wait(&tmem_full_bar[acc], acc_ph, &abort_flag)) {
         atomicOr(p.status, STATUS_TIMEOUT_EPI);
         abort_flag = 1;
       }
