@@ -318,7 +318,16 @@ def run_decode(args, wl):
         torch.cuda.synchronize()
         dev_us = ev0.elapsed_time(ev1) / calls * 1e3
         lory.lory_check_status(ddims, ws)
+        # per-kernel times of a few more calls (events around every launch; not part of the figures above)
+        lory.lory_profile_enable(True)
+        for _ in range(20):
+            lory.lory_moe_ffn(ddims, x_new, None, W1, W2, W3, y_new, ws)
+        per = {}
+        for label, ms in lory.lory_profile_read():
+            per.setdefault(label, []).append(ms * 1e3)
+        lory.lory_profile_enable(False)
         rows.append({"new_tokens_per_sequence": n, "device_us_per_call": dev_us, "host_us_per_call": host_us,
+                     "kernel_us": {k: sum(v) / len(v) for k, v in per.items()},
                      "tokens_per_s": wl.B * n / (dev_us * 1e-6), "launches_per_call": lory.lory_last_launch_count(),
                      "merged_weight_gbs": merged_bytes / (dev_us * 1e-6) / 1e9,
                      "frac_of_hbm_peak": merged_bytes / (dev_us * 1e-6) / 1e9 / peaks["hbm_gbs"]})

@@ -411,15 +411,25 @@ int tc_ffn_forward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* x
   // Y = H Wbar2^T
   {
     CUtensorMap m_h, m_b2, m_y;
-    LORY_TRY(make_map(&m_h, q.H, f, T, S, f, (uint64_t)T * f, 128));
     const bool pair = use_pairs(T);
+    LORY_TRY(make_map(&m_h, q.H, f, T, S, f, (uint64_t)T * f, 128));
+    // Few, short groups (a decode step: a handful of new tokens per sequence): 256-column tiles would leave most
+    // SMs without one while each tile streams a long strip of Wbar2; 64-column tiles spread that read over 4 x the SMs.
+    const bool narrow = !pair && ceil_div(T, 128) * ceil_div(d, 256) * S < sm_count();
     // B tile: 256 rows (n = d index) x 64 cols (k = f index); a CTA pair loads 128 rows each
-    LORY_TRY(make_blocked_map(&m_b2, q.wbar2, d, f, S, 64, 1, 1, pair ? 2 : 4));
+    LORY_TRY(make_blocked_map(&m_b2, q.wbar2, d, f, S, 64, 1, 1, narrow ? 1 : (pair ? 2 : 4)));
     LORY_TRY(make_map(&m_y, y, d, T, S, d, (uint64_t)T * d, 32));
     TcGemmParams p = {};
     p.M = T; p.N = d; p.K = f; p.groups = S; p.status = q.status;
     p.residual = residual;
-    if (residual) {  // y = residual + H Wbar2^T: the block's skip connection rides in the epilogue
+    if (narrow) {
+      if (residual)
+        LORY_TRY((launch_tc<false, false, 64, MODE_PLAIN, EPI_BF16_RESADD, true>("gemm2", m_h, m_h, m_b2, m_b2, m_y, m_y,
+                                                                                  m_y, p, st)));
+      else
+        LORY_TRY((launch_tc<false, false, 64, MODE_PLAIN, EPI_BF16, true>("gemm2", m_h, m_h, m_b2, m_b2, m_y, m_y, m_y,
+                                                                          p, st)));
+    } else if (residual) {  // y = residual + H Wbar2^T: the block's skip connection rides in the epilogue
       if (pair)
         LORY_TRY((launch_tc<false, false, 256, MODE_PLAIN, EPI_BF16_RESADD, true, false, 2>("gemm2", m_h, m_h, m_b2, m_b2,
                                                                                              m_y, m_y, m_y, p, st)));
@@ -444,8 +454,8 @@ int tc_ffn_backward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* 
   // dH = dY Wbar2; dG, dU in the epilogue
   {
     CUtensorMap m_dy, m_b2, m_dgo, m_duo, m_gi, m_ui;
-    LORY_TRY(make_map(&m_dy, dy, d, T, S, d, (uint64_t)T * d, 128));
     const bool pair = use_pairs(T);
+    LORY_TRY(make_map(&m_dy, dy, d, T, S, d, (uint64_t)T * d, 128));
     // B[k = d index (rows), n = f index]: 4 col blocks per tile, 2 per CTA of a pair
     LORY_TRY(make_blocked_map(&m_b2, q.wbar2, d, f, S, 64, 1, pair ? 2 : 4, 1));
     LORY_TRY(make_map(&m_dgo, q.dG, f, T, S, f, (uint64_t)T * f, 128));
@@ -512,9 +522,9 @@ int tc_ffn_backward_dx(const lory_dims& D, const Layout& Lo, char* ws, const flo
   const int S = D.B * (D.L / D.T), T = D.T, d = D.d, f = D.f;
   const WsPtrs q = ws_ptrs(D, Lo, ws);
   CUtensorMap m_dg, m_du, m_b1, m_b3, m_dx;
+  const bool pair = use_pairs(T);
   LORY_TRY(make_map(&m_dg, q.dG, f, T, S, f, (uint64_t)T * f, 128));
   LORY_TRY(make_map(&m_du, q.dU, f, T, S, f, (uint64_t)T * f, 128));
-  const bool pair = use_pairs(T);
   // B[k = f index (rows), n = d index]: 4 col blocks per tile, 2 per CTA of a pair
   LORY_TRY(make_blocked_map(&m_b1, q.wbar1, f, d, S, 64, 1, pair ? 2 : 4, 1));
   LORY_TRY(make_blocked_map(&m_b3, q.wbar3, f, d, S, 64, 1, pair ? 2 : 4, 1));
