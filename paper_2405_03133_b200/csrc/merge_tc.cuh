@@ -1,9 +1,10 @@
 // Expert merging on the tensor cores (Eq. 2):  Wbar_k[s, r, c] = sum_e w[s, e] * W_k[e, r, c],  k = 1, 3, 2.
 //
-// One tile = one matrix row r and 256 consecutive columns, for 128 segments at once:
-//   D[s, 256] = (w_hi + w_lo)[s, E] . W_k[E, (r, c0 .. c0+255)]        (two MMAs per 16 experts)
+// One tile = 256 parameters (1, 2 or 4 neighbouring rows of 256, 128 or 64 consecutive columns), for 128 segments at once:
+//   D[s, 256] = (w_hi + w_lo)[s, E] . W_k[E, 256 parameters]          (two MMAs per 16 experts)
 // The routing weights (bf16 hi + lo, K-major) stay resident in shared memory; each expert tile is
-// loaded once by TMA (4 boxes of 64 columns x E rows) and used for every 128-segment tile.
+// loaded once by TMA (4 boxes of 64 columns x E rows, one per row and column block of the tile) and used for
+// every 128-segment tile.
 // With S <= 64 the segments are placed twice in the 128 rows of the weight tile, and the two copies of the
 // result are split by columns between the epilogue warps.
 // Output goes to the blocked per-segment layout [row block][col block][segment][64][64]: the 128
@@ -28,7 +29,8 @@ struct MergeParams {
   int S, E, Epad16, s_tiles;  // S: segments of this launch (at most 256); s_tiles = ceil(S / 128)
   int seg_base;               // first segment of this launch (launches cover the segments 256 at a time)
   int dup;           // S <= 64: the w maps have 64-row boxes and the 64 segments are placed twice (rows 0..63, 64..127)
-  int ctiles[3];     // 256-column tiles per row
+  int rpt_shift;     // log2 of the rows per tile (1, 2 or 4 rows of 256, 128 or 64 columns)
+  int ctiles[3];     // column tiles per row
   int tile_end[3];   // exclusive prefix sums of rows_padded * ctiles
   int stages, stage_bytes;
   uint32_t* status;
@@ -80,21 +82,26 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
   // tile -> (matrix k, row r, first column c0).  Consecutive tiles walk the 64 rows of one row block for a fixed
   // column tile, so that the CTAs running at the same time fill neighbouring 128-byte pieces of the same output
   // blocks (whole DRAM pages instead of isolated pieces).
+  const int rsh = p.rpt_shift;            // a tile has 1 << rsh rows ...
+  const int cb_per_row = 4 >> rsh;        // ... of this many 64-column blocks each
   auto decode = [&](int tile, int& k, int& r, int& c0) {
     k = tile < p.tile_end[0] ? 0 : (tile < p.tile_end[1] ? 1 : 2);
     const int local = tile - (k == 0 ? 0 : p.tile_end[k - 1]);
-    const int per_rb = 64 * p.ctiles[k];
+    const int per_rb = (64 >> rsh) * p.ctiles[k];
     const int rb = local / per_rb, rem = local - rb * per_rb;
-    r = rb * 64 + (rem & 63);
-    c0 = (rem >> 6) * 256;
+    r = rb * 64 + ((rem & ((64 >> rsh) - 1)) << rsh);
+    c0 = (rem >> (6 - rsh)) * (256 >> rsh);
   };
+  // chunk j of a tile (64 of its 256 accumulator columns): row offset and column-block offset inside the tile
+  auto chunk_row = [&](int j) { return j / cb_per_row; };
+  auto chunk_cb = [&](int j) { return j % cb_per_row; };
 
   // debug build: a decoded tile against the padded tile grid of its matrix
   auto tile_ok = [&](int k, int r, int c0) {
     if (!dbg::kOn) return true;
     if (k < 0 || k > 2) return false;
     const int tiles_k = p.tile_end[k] - (k ? p.tile_end[k - 1] : 0);
-    return dbg::coord_ok(r, tiles_k / p.ctiles[k]) && dbg::inner_ok(c0, p.ctiles[k] * 256);
+    return dbg::coord_ok(r, (tiles_k / p.ctiles[k]) << rsh) && dbg::inner_ok(c0, p.ctiles[k] * (256 >> rsh));
   };
 
   if (warp == 0) {
@@ -132,7 +139,8 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
         issued |= 1u << s;
         last_parity = (last_parity & ~(1u << s)) | (ph << s);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) ptx::tma_load_3d(sB + j * box_bytes, &maps.theta[k], &full_bar[s], c0 + 64 * j, 0, r);
+        for (int j = 0; j < 4; ++j)
+          ptx::tma_load_3d(sB + j * box_bytes, &maps.theta[k], &full_bar[s], c0 + 64 * chunk_cb(j), 0, r + chunk_row(j));
       }
       if (abort_flag) {
         for (int s = 0; s < STAGES; ++s)
@@ -227,7 +235,8 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
           uint8_t* b = warp_stage(wsg, lane, w);
           if (lane == 0) {
             // (col in block, row in block, segment, col block, row block); blocks past the matrix are clipped
-            ptx::tma_store_5d(&maps.out[k], b, 0, r & 63, p.seg_base + st * 128 + seg0, (c0 >> 6) + c, r >> 6);
+            ptx::tma_store_5d(&maps.out[k], b, 0, (r & 63) + chunk_row(c), p.seg_base + st * 128 + seg0,
+                              (c0 >> 6) + chunk_cb(c), r >> 6);
             ptx::tma_store_commit();
           }
           wsg.n++;

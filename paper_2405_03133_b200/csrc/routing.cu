@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(256) pool_kernel(const T* __restrict__ x, floa
 
 // ---------------------------------------------------------------------------------------
 // p_s = softmax(W_r h_bar_s); w_{b,0} = p_{b,0}; w_{b,n} = p_{b,n-1}.
-// One block per segment, one warp per expert in turn.
+// One block per segment; its warps (one per expert when E <= 32) take the experts in turn.
 // ---------------------------------------------------------------------------------------
 // One routing-weight row: fp32 (workspace and, if asked, the caller's copy) and the bf16 hi + lo tables.
 __device__ __forceinline__ void write_weight_row(const float* p_sm, size_t row, int E, int lane, float* w_out,
@@ -114,7 +114,7 @@ __device__ __forceinline__ void write_weight_row(const float* p_sm, size_t row, 
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ h_bar,
+__global__ void __launch_bounds__(1024) router_kernel(const float* __restrict__ h_bar,
                                                      const T* __restrict__ w_r, float* __restrict__ p_ws,
                                                      float* __restrict__ route_p, float* __restrict__ w_out,
                                                      int N, int d, int E, int prefix, const RouteExtra ex) {
@@ -122,7 +122,8 @@ __global__ void __launch_bounds__(256) router_kernel(const float* __restrict__ h
   const int s = blockIdx.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const float* h = h_bar + (size_t)s * d;
-  for (int e = warp; e < E; e += 8) {
+  const int nwarps = blockDim.x >> 5;
+  for (int e = warp; e < E; e += nwarps) {
     const T* wr = w_r + (size_t)e * d;
     float acc = 0.f;
     constexpr int VEC = Vec16<T>::N;
@@ -203,9 +204,18 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(const float* __restrict
   auto reduce_row = [&](size_t row, int mode) {
     for (int e0 = 0; e0 < E; e0 += 128) {
       for (int e = e0 + lane; e < min(E, e0 + 128); e += 32) {
-        float a = 0.f;
-        for (int c = warp; c < n_slabs; c += 8) a += partial[(size_t)c * SE + row * E + e];
-        red[warp][e - e0] = a;
+        // four independent partial sums: the loads of four slabs are in flight together
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        const float* src = partial + row * E + e;
+        int c = warp;
+        for (; c + 24 < n_slabs; c += 32) {
+          a0 += src[(size_t)c * SE];
+          a1 += src[(size_t)(c + 8) * SE];
+          a2 += src[(size_t)(c + 16) * SE];
+          a3 += src[(size_t)(c + 24) * SE];
+        }
+        for (; c < n_slabs; c += 8) a0 += src[(size_t)c * SE];
+        red[warp][e - e0] = (a0 + a1) + (a2 + a3);
       }
       __syncthreads();
       for (int e = e0 + threadIdx.x; e < min(E, e0 + 128); e += 256) {
@@ -249,40 +259,86 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(const float* __restrict
     }
   }
   __syncthreads();
-  for (int j = threadIdx.x; j < d; j += blockDim.x) {
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    int e = 0;
-    for (; e + 3 < E; e += 4) {
-      a0 += dz_sm[e] * to_f32(w_r[(size_t)e * d + j]);
-      a1 += dz_sm[e + 1] * to_f32(w_r[(size_t)(e + 1) * d + j]);
-      a2 += dz_sm[e + 2] * to_f32(w_r[(size_t)(e + 2) * d + j]);
-      a3 += dz_sm[e + 3] * to_f32(w_r[(size_t)(e + 3) * d + j]);
+  // dh_bar_s = W_r^T dz_s.  A thread takes VEC consecutive columns (one 16-byte load per expert row) and one
+  // half of the experts; the two halves of the block meet in shared memory.  All loads of a thread are independent.
+  constexpr int VEC = Vec16<T>::N;
+  if (d % VEC == 0) {
+    float* xch = &red[0][0];  // 128 threads x VEC <= 1024 floats
+    const int nvec = d / VEC, half = threadIdx.x >> 7, vt = threadIdx.x & 127;
+    const int eh = (E + 1) / 2, e_begin = half * eh, e_end = min(E, e_begin + eh);
+    for (int v0 = 0; v0 < nvec; v0 += 128) {
+      const int v = v0 + vt;
+      float acc[VEC];
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
+      if (v < nvec) {
+#pragma unroll 8
+        for (int e = e_begin; e < e_end; ++e) {
+          float wv[VEC];
+          Vec16<T>::load(w_r + (size_t)e * d + (size_t)v * VEC, wv);
+          const float z = dz_sm[e];
+#pragma unroll
+          for (int i = 0; i < VEC; ++i) acc[i] += z * wv[i];
+        }
+      }
+      if (half == 1) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) xch[i * 128 + vt] = acc[i];
+      }
+      __syncthreads();
+      if (half == 0 && v < nvec) {
+#pragma unroll
+        for (int i = 0; i < VEC; i += 4) {
+          float4 o = make_float4(acc[i] + xch[i * 128 + vt], acc[i + 1] + xch[(i + 1) * 128 + vt],
+                                 acc[i + 2] + xch[(i + 2) * 128 + vt], acc[i + 3] + xch[(i + 3) * 128 + vt]);
+          *reinterpret_cast<float4*>(dh_bar + (size_t)s * d + (size_t)v * VEC + i) = o;
+        }
+      }
+      __syncthreads();
     }
-    for (; e < E; ++e) a0 += dz_sm[e] * to_f32(w_r[(size_t)e * d + j]);
-    dh_bar[(size_t)s * d + j] = (a0 + a1) + (a2 + a3);
+  } else {
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+      float a0 = 0.f;
+      for (int e = 0; e < E; ++e) a0 += dz_sm[e] * to_f32(w_r[(size_t)e * d + j]);
+      dh_bar[(size_t)s * d + j] = a0;
+    }
   }
 }
 
-// dW_r[e, j] = sum_s dz[s,e] h_bar[s,j].  grid (ceil(d/256), E).
+// dW_r[e, j] = sum_s dz[s,e] h_bar[s,j].  grid (ceil(d/64), ceil(E/4)), block 512 = 64 columns x 8 runs of
+// segments: a thread sums its run for one column and four experts (each h_bar element it loads serves the four),
+// then the eight runs are added in a fixed order through shared memory.
 template <typename T>
-__global__ void __launch_bounds__(256) dwr_kernel(const float* __restrict__ dz, const float* __restrict__ h_bar,
+__global__ void __launch_bounds__(512) dwr_kernel(const float* __restrict__ dz, const float* __restrict__ h_bar,
                                                   T* __restrict__ dw_r, int S, int d, int E, int accumulate) {
-  const int e = blockIdx.y;
-  const int j = blockIdx.x * 256 + threadIdx.x;
-  if (j >= d) return;
-  // four independent partial sums keep several loads in flight
-  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-  int s = 0;
-  for (; s + 3 < S; s += 4) {
-    a0 += dz[(size_t)s * E + e] * h_bar[(size_t)s * d + j];
-    a1 += dz[(size_t)(s + 1) * E + e] * h_bar[(size_t)(s + 1) * d + j];
-    a2 += dz[(size_t)(s + 2) * E + e] * h_bar[(size_t)(s + 2) * d + j];
-    a3 += dz[(size_t)(s + 3) * E + e] * h_bar[(size_t)(s + 3) * d + j];
+  __shared__ float red[8][4][64];
+  const int jj = threadIdx.x & 63, part = threadIdx.x >> 6;
+  const int j = blockIdx.x * 64 + jj, e0 = blockIdx.y * 4;
+  const int run = (S + 7) / 8;
+  const int s_begin = part * run, s_end = min(S, s_begin + run);
+  float a[4] = {0.f, 0.f, 0.f, 0.f};
+  if (j < d) {
+#pragma unroll 4
+    for (int s = s_begin; s < s_end; ++s) {
+      const float h = h_bar[(size_t)s * d + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (e0 + i < E) a[i] += dz[(size_t)s * E + e0 + i] * h;
+    }
   }
-  for (; s < S; ++s) a0 += dz[(size_t)s * E + e] * h_bar[(size_t)s * d + j];
-  float out = (a0 + a1) + (a2 + a3);
-  if (accumulate) out += to_f32(dw_r[(size_t)e * d + j]);
-  dw_r[(size_t)e * d + j] = from_f32<T>(out);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) red[part][i][jj] = a[i];
+  __syncthreads();
+  if (threadIdx.x < 256) {
+    const int i = threadIdx.x >> 6, e = e0 + i;
+    if (j < d && e < E) {
+      float out = 0.f;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) out += red[q][i][jj];
+      if (accumulate) out += to_f32(dw_r[(size_t)e * d + j]);
+      dw_r[(size_t)e * d + j] = from_f32<T>(out);
+    }
+  }
 }
 
 // dx[t, j] += dh_bar[s(t), j] / T   (mean-pool backward), fp32 add then round to storage.
@@ -308,7 +364,8 @@ int launch_pool_router(const T* x, const T* w_r, float* h_bar, float* p_ws, floa
   dim3 grid(S, (unsigned)ceil_div(d, 32 * VEC));
   pool_kernel<T><<<grid, 256, 0, st>>>(x, h_bar, Tseg, d);
   LORY_AFTER_LAUNCH();
-  router_kernel<T><<<S, 256, E * sizeof(float), st>>>(h_bar, w_r, p_ws, route_p, w_out, N, d, E, prefix, extra);
+  const int router_threads = E >= 32 ? 1024 : (E > 8 ? 32 * E : 256);  // one warp per expert, 8 to 32 warps
+  router_kernel<T><<<S, router_threads, E * sizeof(float), st>>>(h_bar, w_r, p_ws, route_p, w_out, N, d, E, prefix, extra);
   LORY_AFTER_LAUNCH();
   return LORY_OK;
 }
@@ -320,7 +377,7 @@ int launch_router_backward(const float* dw_partial, int n_slabs, const float* p_
   const int S = B * N;
   router_bwd_kernel<T><<<S, 256, 2 * E * sizeof(float), st>>>(dw_partial, n_slabs, p_ws, w_r, dw, d_route_w, dz, dh_bar, S, N, d, E, prefix);
   LORY_AFTER_LAUNCH();
-  dwr_kernel<T><<<dim3((unsigned)ceil_div(d, 256), E), 256, 0, st>>>(dz, h_bar, dw_r, S, d, E, (prefix & 4) ? 1 : 0);
+  dwr_kernel<T><<<dim3((unsigned)ceil_div(d, 64), (unsigned)ceil_div(E, 4)), 512, 0, st>>>(dz, h_bar, dw_r, S, d, E, (prefix & 4) ? 1 : 0);
   LORY_AFTER_LAUNCH();
   return LORY_OK;
 }

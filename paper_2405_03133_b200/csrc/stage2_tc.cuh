@@ -32,7 +32,8 @@ struct Stage2Maps {
 struct Stage2Params {
   int S, E, Epad16, s_tiles;  // S: segments of this launch (at most 256); s_tiles = ceil(S / 128)
   int seg_base, S_total;      // first segment of this launch; all segments (row count of a dw slab)
-  int ctiles[3];    // 128-column tiles per row
+  int rpt_shift;    // 0: a tile is 128 columns of one row; 1: 64 columns of two neighbouring rows
+  int ctiles[3];    // column tiles per row
   uint32_t cmagic[3];  // ceil(2^32 / ctiles), 0 for ctiles == 1: n / ctiles == __umulhi(n, cmagic) for every tile index n
   int tile_end[3];  // exclusive prefix sums of (rows rounded up to 64) * ctiles
   int cb_stride;    // bytes between the two 64-column blocks of a dWbar tile in shared memory (= segments per box * 128)
@@ -74,15 +75,18 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
     const int local = tile - (k == 0 ? 0 : p.tile_end[k - 1]);
     // local / ctiles[k] without the division (a single tile per row has no 32-bit reciprocal: magic 0)
     r = p.cmagic[k] ? (int)__umulhi((uint32_t)local, p.cmagic[k]) : local;
-    c0 = (local - r * p.ctiles[k]) * 128;
+    c0 = (local - r * p.ctiles[k]) * (128 >> p.rpt_shift);
+    r <<= p.rpt_shift;
   };
+  // the two 64-column halves of a tile: columns c0 and c0 + 64 of row r, or (two-row tiles) column c0 of rows r, r + 1
+  const int half_col = p.rpt_shift ? 0 : 64, half_row = p.rpt_shift ? 1 : 0;
 
   // debug build: a decoded tile against the padded tile grid of its matrix
   auto tile_ok = [&](int k, int r, int c0) {
     if (!dbg::kOn) return true;
     if (k < 0 || k > 2) return false;
     const int tiles_k = p.tile_end[k] - (k ? p.tile_end[k - 1] : 0);
-    return dbg::coord_ok(r, tiles_k / p.ctiles[k]) && dbg::inner_ok(c0, p.ctiles[k] * 128);
+    return dbg::coord_ok(r, (tiles_k / p.ctiles[k]) << p.rpt_shift) && dbg::inner_ok(c0, p.ctiles[k] * (128 >> p.rpt_shift));
   };
 
   if (threadIdx.x == 0) {
@@ -143,9 +147,15 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           issued |= 1u << s;
           last_parity = (last_parity & ~(1u << s)) | (ph << s);
           // (col in block, row in block, segment, col block, row block): two col blocks, 128 segments
-          ptx::tma_load_5d(sD, &maps.dwbar[k], &full_bar[s], 0, r & 63, p.seg_base + st * 128, c0 >> 6, r >> 6);
+          if (p.rpt_shift) {  // two boxes of one column block each (rows r, r + 1)
+            ptx::tma_load_5d(sD, &maps.dwbar[k], &full_bar[s], 0, r & 63, p.seg_base + st * 128, c0 >> 6, r >> 6);
+            ptx::tma_load_5d(sD + p.cb_stride, &maps.dwbar[k], &full_bar[s], 0, (r & 63) + 1, p.seg_base + st * 128,
+                             c0 >> 6, r >> 6);
+          } else {            // one box of two column blocks
+            ptx::tma_load_5d(sD, &maps.dwbar[k], &full_bar[s], 0, r & 63, p.seg_base + st * 128, c0 >> 6, r >> 6);
+          }
           ptx::tma_load_3d(sT, &maps.theta[k], &full_bar[s], c0, 0, r);
-          ptx::tma_load_3d(sT + p.Epad16 * 128, &maps.theta[k], &full_bar[s], c0 + 64, 0, r);
+          ptx::tma_load_3d(sT + p.Epad16 * 128, &maps.theta[k], &full_bar[s], c0 + half_col, 0, r + half_row);
         }
       }
       if (abort_flag) {
@@ -296,9 +306,9 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           // the tile leaves the tensor
           uint4 old[8];
           if (ACC) {
-            const int e = e0 + lane, col0 = c0 + c * 64;
-            const bool row_ok = e < p.E && row < p.rows[k];
-            const __nv_bfloat16* src = p.acc_base[k] + ((size_t)e * p.rows[k] + row) * p.cols[k] + col0;
+            const int e = e0 + lane, col0 = c0 + c * half_col, rowc = row + c * half_row;
+            const bool row_ok = e < p.E && rowc < p.rows[k];
+            const __nv_bfloat16* src = p.acc_base[k] + ((size_t)e * p.rows[k] + rowc) * p.cols[k] + col0;
 #pragma unroll
             for (int j = 0; j < 8; ++j)
               old[j] = (row_ok && col0 + 8 * j < p.cols[k]) ? *reinterpret_cast<const uint4*>(src + 8 * j)
@@ -329,7 +339,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
             ptx::tc_fence_before_sync();
             ptx::mbar_arrive(&tmem_empty_bar[acc]);
           }
-          warp_stage_and_store(wsg, &maps.out[k], c0 + c * 64, e0, row, lane, w);
+          warp_stage_and_store(wsg, &maps.out[k], c0 + c * half_col, e0, row + c * half_row, lane, w);
         }
       }
     }
