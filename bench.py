@@ -26,6 +26,9 @@ METRIC = "Lory MoE-layer fwd+bwd tokens/s (bf16, 1 B200)"
 UNIT = "tokens/s"
 
 
+PROF_RECORDS = 8192   # capacity of the library's per-launch event table
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -348,6 +351,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-sustained", action="store_true", help="skip the second timed region of >= 1 s")
+    ap.add_argument("--chunked-adjoint", action="store_true",
+                    help="A/B: run the backward with LORY_FLAG_CHUNKED_ADJOINT (per-segment weight gradients kept in "
+                         "an L2-sized buffer, one parameter rectangle at a time) instead of the default")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture one forward+backward (the same C-ABI calls) in a CUDA graph and time its replays: "
+                         "takes the host's launch work out of the picture")
     ap.add_argument("--decode", action="store_true",
                     help="measure the inference path instead: prefill with prompt-only routing, then decode calls")
     args = ap.parse_args()
@@ -391,7 +400,8 @@ def main():
     W2 = normal((wl.E, wl.d, wl.f), 0.02)
     W3 = normal((wl.E, wl.f, wl.d), 0.02)
     dy = normal((wl.B, wl.L, wl.d), 1.0)
-    dims = lory.make_dims(wl.B, wl.L, wl.T, wl.d, wl.f, wl.E, "bf16")
+    dims = lory.make_dims(wl.B, wl.L, wl.T, wl.d, wl.f, wl.E, "bf16",
+                          lory.LORY_FLAG_CHUNKED_ADJOINT if args.chunked_adjoint else 0)
     _, bwd_bytes = lory.lory_moe_workspace_bytes(dims)
     ws = torch.empty(bwd_bytes, dtype=torch.uint8, device=dev)
     y = torch.empty_like(x)
@@ -401,12 +411,27 @@ def main():
     dW1, dW2, dW3 = torch.empty_like(W1), torch.empty_like(W2), torch.empty_like(W3)
 
     launches = [0]
+    # a stream of our own: the calls below name it, the events of the timed region are recorded on it
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(stream)
+    sp = stream.cuda_stream
 
-    def step():
-        lory.lory_moe_forward(dims, x, w_r, W1, W2, W3, y, route_w, None, ws)
+    def step_calls():
+        lory.lory_moe_forward(dims, x, w_r, W1, W2, W3, y, route_w, None, ws, stream=sp)
         n = lory.lory_last_launch_count()
-        lory.lory_moe_backward(dims, x, w_r, W1, W2, W3, dy, dx, dw_r, dW1, dW2, dW3, None, ws)
+        lory.lory_moe_backward(dims, x, w_r, W1, W2, W3, dy, dx, dw_r, dW1, dW2, dW3, None, ws, stream=sp)
         launches[0] = n + lory.lory_last_launch_count()
+
+    step = step_calls
+    if args.graph:
+        for _ in range(2):          # first calls set per-device function attributes: not inside a capture
+            step_calls()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            step_calls()
+        torch.cuda.set_stream(stream)
+        step = graph.replay
 
     def barrier():
         if dist is not None:
@@ -418,14 +443,17 @@ def main():
     lory.lory_check_status(dims, ws)
     barrier()
 
-    def timed_region(n_steps):
-        """n_steps back to back, device-resident inputs, CUDA events on the launch stream around the whole region
-        and (through the library's profiling hooks) around every kernel; SM clocks sampled meanwhile."""
+    def timed_region(n_steps, per_kernel=False, settle=True):
+        """n_steps back to back, device-resident inputs, CUDA events on the launch stream around the whole region;
+        SM clocks sampled meanwhile.  per_kernel: the library's profiling hooks also put an event pair around every
+        kernel (26 events per step, which cost 2-3 % of the step: the headline region runs without them).
+        settle=False: no pause before the region (it follows another one and should see the same clocks)."""
         sampler = ClockSampler(local_rank)
         if rank == 0:
             sampler.start()
-            time.sleep(0.3)
-        lory.lory_profile_enable(True)
+            if settle:
+                time.sleep(0.3)
+        lory.lory_profile_enable(per_kernel and not args.graph)   # a replayed graph holds no per-kernel events
         barrier()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_wall0 = time.time()
@@ -441,8 +469,10 @@ def main():
         lory.lory_check_status(dims, ws)
         return ms, recs, (sampler.stop(t_wall0, t_wall1) if rank == 0 else None)
 
-    ms_total, records, clocks = timed_region(args.steps)
+    ms_total, _, clocks = timed_region(args.steps)
     ms_per_step, value = aggregate_over_ranks(ms_total, args.steps, wl.tokens, world, dist, dev)
+    # the same K steps once more with an event pair around every kernel: per-kernel times and shares
+    ms_prof, records, clocks_prof = timed_region(args.steps, per_kernel=True)
 
     peaks = load_peaks()
     # Which measured tensor peak a run is compared with: the burst figure while the SM clock stays near its maximum
@@ -484,7 +514,7 @@ def main():
             out[label] = ent
         return out
 
-    kernels = kernel_stats(records, args.steps, clocks)
+    kernels = kernel_stats(records, args.steps, clocks_prof)
     reg_name, tensor_peak = regime(clocks)
     top = max(kernels, key=lambda k: kernels[k]["share"]) if kernels else None
     roofline = None
@@ -521,10 +551,13 @@ def main():
     sustained = None
     if not args.no_sustained:
         n_long = max(400, int(1.2e3 / ms_per_step))
-        ms_long, rec_long, clk_long = timed_region(n_long)
+        ms_long, _, clk_long = timed_region(n_long)
         ms_step_long, value_long = aggregate_over_ranks(ms_long, n_long, wl.tokens, world, dist, dev)
         tf_long = F / (ms_step_long * 1e-3) / 1e12
-        k_long = kernel_stats(rec_long, n_long, clk_long)
+        # per-kernel times in the same regime: a shorter instrumented region straight after it
+        n_k = min(100, PROF_RECORDS // max(1, launches[0]))
+        _, rec_long, clk_k = timed_region(n_k, per_kernel=True, settle=False)
+        k_long = kernel_stats(rec_long, n_k, clk_k)
         sustained = {"steps": n_long, "ms_per_step": ms_step_long, "value": value_long, "unit": UNIT,
                      "clocks": clk_long, "achieved_tflops": tf_long,
                      "frac_of_sustained_peak": tf_long / peaks["bf16_tflops_sustained"],
@@ -606,10 +639,17 @@ def main():
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic", "config": workload_config(wl), "clocks": clocks, "e2e": e2e,
+        "dtype": "bf16", "data": "synthetic",
+        "config": dict(workload_config(wl), **({"backward": "chunked adjoint (LORY_FLAG_CHUNKED_ADJOINT), workspace "
+                                                f"{bwd_bytes / 1e9:.2f} GB"} if args.chunked_adjoint else {})),
+        "clocks": clocks, "e2e": e2e,
         "gpu_launches": launches[0] * args.steps, "roofline": roofline, "cpu_baseline": cpu, "layer": layer,
         "sustained": sustained, "kernels": kernels,
+        "kernels_note": "per-kernel times come from a second region of the same K steps with a CUDA-event pair "
+                        f"around every launch ({ms_prof / args.steps:.3f} ms per step with them)",
     }
+    if args.graph:
+        out["config"]["launch"] = "one CUDA graph per step (the captured C-ABI calls), replayed"
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()

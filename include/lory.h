@@ -68,6 +68,16 @@ typedef enum { LORY_FP32 = 0, LORY_BF16 = 1 } lory_dtype;
                                          the gradient (micro-batches of one optimiser step; the sum is formed in
                                          fp32 and rounded to the storage type).  dx and d_route_w are per call. */
 
+#define LORY_FLAG_CHUNKED_ADJOINT 32 /* backward only, tensor-core pipeline: the per-segment weight gradients (the
+                                        adjoint of Eq. 2 needs them for every segment) are formed one rectangle of
+                                        one expert matrix at a time in a buffer sized to half the device's L2 and
+                                        consumed from there, instead of being written out for the whole matrices.
+                                        Same results up to the summation order of the routing gradient; the
+                                        backward workspace shrinks by almost the size of the merged weights (2.1 GB
+                                        at E = 32, T = 256, d = 1024, f = 2752); about twice the launches of the
+                                        default backward and slower (measurements in the design notes).  Ignored
+                                        by the plain-FMA pipeline.  Pass it to lory_moe_workspace_bytes as well. */
+
 /*
  * Problem description.  B sequences of L tokens, segment length T (L % T == 0),
  * hidden size d, FFN hidden size f, E experts.

@@ -16,6 +16,7 @@ LORY_FLAG_REUSE_MERGED = 2
 LORY_FLAG_PREFIX_ROUTING = 4
 LORY_FLAG_FIRST_SEGMENT_GRAD = 8
 LORY_FLAG_ACCUMULATE_GRADS = 16
+LORY_FLAG_CHUNKED_ADJOINT = 32
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 # LORY_LIBRARY selects another build of the same ABI, e.g. the bounds-checking liblory_debug.so

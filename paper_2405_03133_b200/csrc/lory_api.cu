@@ -94,9 +94,15 @@ static Layout make_layout(const lory_dims& D) {
   Lo.fwd_end = off;
   Lo.dG = take(tok * D.f * es);
   Lo.dU = take(tok * D.f * es);
-  Lo.dwbar1 = take(n13 * es);
-  Lo.dwbar3 = take(n13 * es);
-  Lo.dwbar2 = take(n2 * es);
+  if (blk && (D.flags & LORY_FLAG_CHUNKED_ADJOINT)) {
+    // one L2-sized buffer for a rectangle of per-segment weight gradients at a time
+    Lo.dwbar1 = take(tc_adjoint_ring_elems(D) * es);
+    Lo.dwbar3 = Lo.dwbar2 = Lo.dwbar1;
+  } else {
+    Lo.dwbar1 = take(n13 * es);
+    Lo.dwbar3 = take(n13 * es);
+    Lo.dwbar2 = take(n2 * es);
+  }
   Lo.k_chunk = 8192;
   int simt_slabs = 3 * (int)ceil_div((long)P1, Lo.k_chunk);
   Lo.n_slabs = use_tc(D) ? tc_dw_slabs(D) : simt_slabs;

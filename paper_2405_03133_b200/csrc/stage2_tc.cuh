@@ -41,9 +41,11 @@ struct Stage2Params {
   int xch_bytes;    // one exchange buffer: 32 lanes x 256 B, or x 128 B with E <= 32
   int stages;       // pipeline depth (<= 8)
   int stage_bytes, tx_bytes;
-  const __nv_bfloat16* acc_base[3];  // the three output tensors [E, rows, cols], read by the accumulating variant
-  int rows[3], cols[3];
-  float* dw_partial;  // [gridDim.x, S, E]
+  const __nv_bfloat16* acc_base[3];  // the three output tensors (or sub-rectangles of them), read by the accumulating variant
+  int rows[3], cols[3];              // extent of each
+  long e_stride[3], row_stride[3];   // elements between experts and between rows of each
+  int slab_add;       // add to the dw slab instead of overwriting it (a launch that covers part of the parameters)
+  float* dw_partial;  // [slabs, S, E]; CTA b owns slab b
   uint32_t* status;
 };
 
@@ -308,7 +310,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           if (ACC) {
             const int e = e0 + lane, col0 = c0 + c * half_col, rowc = row + c * half_row;
             const bool row_ok = e < p.E && rowc < p.rows[k];
-            const __nv_bfloat16* src = p.acc_base[k] + ((size_t)e * p.rows[k] + rowc) * p.cols[k] + col0;
+            const __nv_bfloat16* src = p.acc_base[k] + (size_t)e * p.e_stride[k] + (size_t)rowc * p.row_stride[k] + col0;
 #pragma unroll
             for (int j = 0; j < 8; ++j)
               old[j] = (row_ok && col0 + 8 * j < p.cols[k]) ? *reinterpret_cast<const uint4*>(src + 8 * j)
@@ -361,7 +363,10 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
         if (srow < p.S) {
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (c * 32 + j < p.E) slab[(size_t)srow * p.E + c * 32 + j] = __uint_as_float(r[j]);
+            if (c * 32 + j < p.E) {
+              float* dst = slab + (size_t)srow * p.E + c * 32 + j;
+              *dst = p.slab_add ? *dst + __uint_as_float(r[j]) : __uint_as_float(r[j]);
+            }
         }
       }
     }

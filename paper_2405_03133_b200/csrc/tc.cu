@@ -14,6 +14,7 @@
 
 #include <cuda.h>
 #include <stdio.h>
+#include <stdlib.h>
 
 #include "gemm_tc.cuh"
 #include "merge_tc.cuh"
@@ -97,9 +98,11 @@ static int make_blocked_map(CUtensorMap* m, const void* base, int R, int C, int 
 }
 
 // Expert matrix W_k [E, R, C] seen as (C, E, R): a box is 64 columns x box_e experts of one row.
-static int make_expert_map(CUtensorMap* m, const void* base, int R, int C, int E, uint32_t box_e) {
+// e_stride / row_stride (elements) describe a sub-rectangle of a larger [E, R0, C0] tensor; 0 = dense [E, R, C].
+static int make_expert_map(CUtensorMap* m, const void* base, int R, int C, int E, uint32_t box_e, uint64_t e_stride = 0,
+                           uint64_t row_stride = 0) {
   const uint64_t dims[3] = {(uint64_t)C, (uint64_t)E, (uint64_t)R};
-  const uint64_t strides[2] = {(uint64_t)R * C, (uint64_t)C};
+  const uint64_t strides[2] = {e_stride ? e_stride : (uint64_t)R * C, row_stride ? row_stride : (uint64_t)C};
   const uint32_t box[3] = {64, box_e, 1};
   return make_map_nd(m, base, 3, dims, strides, box);
 }
@@ -225,23 +228,82 @@ size_t tc_blocked_elems(const lory_dims& D, int R, int C) {
 static int stage2_rpt_shift(const lory_dims& D) {
   return D.B * (D.L / D.T) <= 32 ? 1 : 0;
 }
-static void stage2_tiles(const lory_dims& D, int ctiles[3], int tile_end[3]) {
-  const int R[3] = {D.f, D.f, D.d}, C[3] = {D.d, D.d, D.f};
+// One of the (up to three) parameter rectangles a launch of the merge adjoint covers: a whole expert matrix, or a
+// sub-rectangle of one whose per-segment gradients sit in a buffer of their own.  R == 0: not part of the launch.
+struct AdjPiece {
+  const bf16* dsrc;  // blocked per-segment gradients of the rectangle [R, C]
+  const bf16* wsrc;  // experts: first element of the rectangle inside W_k
+  bf16* ddst;        // expert gradients: first element of the rectangle inside dW_k
+  int R, C;
+  uint64_t e_stride, row_stride;  // elements between experts / rows of W_k and dW_k
+};
+static void stage2_tiles(const lory_dims& D, const int R[3], const int C[3], int ctiles[3], int tile_end[3]) {
   const int rsh = stage2_rpt_shift(D);
   int acc = 0;
   for (int k = 0; k < 3; ++k) {
-    ctiles[k] = (C[k] + (128 >> rsh) - 1) / (128 >> rsh);
+    ctiles[k] = C[k] > 0 ? (C[k] + (128 >> rsh) - 1) / (128 >> rsh) : 1;
     acc += (((R[k] + 63) / 64 * 64) >> rsh) * ctiles[k];  // whole row blocks: the rows past R[k] read zeros and store nothing
     tile_end[k] = acc;
   }
 }
 static int stage2_grid(const lory_dims& D) {
+  const int R[3] = {D.f, D.f, D.d}, C[3] = {D.d, D.d, D.f};
   int ct[3], te[3];
-  stage2_tiles(D, ct, te);
+  stage2_tiles(D, R, C, ct, te);
   return te[2] < sm_count() ? te[2] : sm_count();
 }
 
 int tc_dw_slabs(const lory_dims& D) { return stage2_grid(D); }
+
+// ---------------------------------------------------------------------------------------
+// Chunked adjoint (LORY_FLAG_CHUNKED_ADJOINT): the per-segment weight gradients of one rectangle of one expert
+// matrix at a time (all segments), written by the weight-gradient GEMM into a buffer small enough to stay in L2
+// and consumed from there by the merge adjoint before the next rectangle overwrites it.
+// ---------------------------------------------------------------------------------------
+static size_t adjoint_budget_bytes() {
+  // read on every call: the workspace query and the backward must see the same value, nothing else is assumed
+  if (const char* ev = getenv("LORY_ADJOINT_CHUNK_MB")) {
+    const long mb = atol(ev);
+    if (mb > 0) return (size_t)mb << 20;
+  }
+  static size_t bytes[kMaxDevices];
+  const int dev = current_device();
+  if (!bytes[dev]) {
+    int l2 = 0;
+    if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess || l2 <= 0) l2 = 64 << 20;
+    bytes[dev] = (size_t)l2 / 2;  // what a producer can leave in L2 for the consumer that follows it
+  }
+  return bytes[dev];
+}
+struct AdjChunks {
+  int rows;     // rows of a rectangle (256: one row of CTA-pair tiles; fewer for small matrices)
+  int cols[3];  // columns of a rectangle of W1 / W3 / W2, a multiple of 256 (or the whole width)
+};
+static AdjChunks adjoint_chunks(const lory_dims& D) {
+  const size_t S = (size_t)D.B * (D.L / D.T);
+  const int R[3] = {D.f, D.f, D.d}, C[3] = {D.d, D.d, D.f};
+  AdjChunks a;
+  a.rows = 256;
+  const size_t per_col = (size_t)a.rows * S * 2;  // bytes of one column of a rectangle over all segments
+  long cmax = (long)(adjoint_budget_bytes() / per_col) / 256 * 256;
+  if (cmax < 256) cmax = 256;
+  for (int k = 0; k < 3; ++k) {
+    (void)R;
+    const long n = ceil_div(C[k], cmax);
+    a.cols[k] = (int)(ceil_div(ceil_div(C[k], n), 256) * 256);
+  }
+  return a;
+}
+size_t tc_adjoint_ring_elems(const lory_dims& D) {
+  const AdjChunks a = adjoint_chunks(D);
+  const size_t S = (size_t)D.B * (D.L / D.T);
+  size_t best = 0;
+  for (int k = 0; k < 3; ++k) {
+    const size_t e = (size_t)(a.rows / 64) * (size_t)((a.cols[k] + 63) / 64) * S * 4096;
+    if (e > best) best = e;
+  }
+  return best;
+}
 
 // CTA pairs (256-row tiles) pay off when a segment fills them.
 static bool use_pairs(int rows) { return rows % 256 == 0; }
@@ -313,18 +375,25 @@ static int launch_merge(const lory_dims& D, const WsPtrs& q, const bf16* const s
   return LORY_OK;
 }
 
-// dW_k = w^T dWbar_k and the dw partial slabs, one pass over the blocked dWbar_k
-static int launch_stage2(const lory_dims& D, const WsPtrs& q, const bf16* const dsrc[3], const bf16* const wsrc[3],
-                         bf16* const ddst[3], cudaStream_t st) {
+// dW_k = w^T dWbar_k and the dw partial slabs, one pass over the blocked dWbar_k of every piece.
+// slab_add: the launch covers only part of the parameters, so its dw sums are added to the slabs.
+static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[3], bool slab_add, cudaStream_t st) {
   const int S = D.B * (D.L / D.T), E = D.E, Ep = e_pad(D);
-  const int R[3] = {D.f, D.f, D.d}, C[3] = {D.d, D.d, D.f};
+  int R[3], C[3], first = -1;
+  for (int k = 0; k < 3; ++k) {
+    R[k] = pc[k].R;
+    C[k] = pc[k].R > 0 ? pc[k].C : 0;
+    if (R[k] > 0 && first < 0) first = k;
+  }
+  if (first < 0) return LORY_OK;
   Stage2Maps maps;
   Stage2Params p = {};
   const int S_launch = S < 256 ? S : 256;
   p.S = S_launch; p.S_total = S; p.E = E; p.Epad16 = e_pad16(D); p.s_tiles = (S_launch + 127) / 128;
   p.dw_partial = q.dw_partial; p.status = q.status;
+  p.slab_add = slab_add ? 1 : 0;
   p.rpt_shift = stage2_rpt_shift(D);
-  stage2_tiles(D, p.ctiles, p.tile_end);
+  stage2_tiles(D, R, C, p.ctiles, p.tile_end);
   for (int k = 0; k < 3; ++k)
     p.cmagic[k] = p.ctiles[k] == 1 ? 0u : (uint32_t)(((1ull << 32) + p.ctiles[k] - 1) / p.ctiles[k]);
   if ((uint64_t)p.tile_end[2] * 64 >= (1ull << 32)) return LORY_ERR_SHAPE;  // keeps the reciprocal division exact
@@ -341,12 +410,15 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const bf16* const 
     LORY_TRY(make_map(&maps.w_lo, q.w_lo, Ep, S, 1, Ep, 0, 128));
   }
   for (int k = 0; k < 3; ++k) {
-    LORY_TRY(make_blocked_map(&maps.dwbar[k], dsrc[k], R[k], C[k], S, 1, seg_box, p.rpt_shift ? 1 : 2, 1));
-    LORY_TRY(make_expert_map(&maps.theta[k], wsrc[k], R[k], C[k], E, p.Epad16));
-    LORY_TRY(make_expert_map(&maps.out[k], ddst[k], R[k], C[k], E, 32));
-    p.acc_base[k] = ddst[k];
-    p.rows[k] = R[k];
-    p.cols[k] = C[k];
+    const AdjPiece& a = pc[R[k] > 0 ? k : first];  // an absent piece has no tiles; its maps repeat a present one
+    LORY_TRY(make_blocked_map(&maps.dwbar[k], a.dsrc, a.R, a.C, S, 1, seg_box, p.rpt_shift ? 1 : 2, 1));
+    LORY_TRY(make_expert_map(&maps.theta[k], a.wsrc, a.R, a.C, E, p.Epad16, a.e_stride, a.row_stride));
+    LORY_TRY(make_expert_map(&maps.out[k], a.ddst, a.R, a.C, E, 32, a.e_stride, a.row_stride));
+    p.acc_base[k] = a.ddst;
+    p.rows[k] = a.R;
+    p.cols[k] = a.C;
+    p.e_stride[k] = (long)a.e_stride;
+    p.row_stride[k] = (long)a.row_stride;
   }
   p.stage_bytes = 2 * p.cb_stride + 2 * p.Epad16 * 128;  // dWbar tile (two 64-column blocks) + expert tile
   p.tx_bytes = p.stage_bytes;
@@ -361,6 +433,7 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const bf16* const 
   static bool attr_set[2][kMaxDevices];
   LORY_TRY(allow_dynamic_smem(stage2_kernel<false>, kMaxSmem, attr_set[0]));
   LORY_TRY(allow_dynamic_smem(stage2_kernel<true>, kMaxSmem, attr_set[1]));
+  const int grid = p.tile_end[2] < sm_count() ? p.tile_end[2] : sm_count();
   // One launch per 256 segments; launches after the first add to the expert gradients the earlier ones stored
   // (the same read-add-store as gradient accumulation), and each writes its own rows of the dw slabs.
   for (int base = 0; base < S; base += 256) {
@@ -368,8 +441,8 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const bf16* const 
     p.S = S - base < 256 ? S - base : 256;
     p.s_tiles = (p.S + 127) / 128;
     ProfScope ps("stage2", st);
-    if (base > 0 || (D.flags & LORY_FLAG_ACCUMULATE_GRADS)) stage2_kernel<true><<<stage2_grid(D), 192, smem, st>>>(maps, p);
-    else stage2_kernel<false><<<stage2_grid(D), 192, smem, st>>>(maps, p);
+    if (base > 0 || (D.flags & LORY_FLAG_ACCUMULATE_GRADS)) stage2_kernel<true><<<grid, 192, smem, st>>>(maps, p);
+    else stage2_kernel<false><<<grid, 192, smem, st>>>(maps, p);
     LORY_AFTER_LAUNCH();
   }
   return LORY_OK;
@@ -457,6 +530,49 @@ int tc_ffn_forward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* x
   return LORY_OK;
 }
 
+// Weight gradients and merge adjoint, one parameter rectangle at a time through the ring (see adjoint_chunks).
+// Per rectangle: dWbar_k[rect] = A^T B over every segment (K = T) into the ring, then dW_k[rect] = w^T dWbar_k[rect]
+// and the rectangle's share of dw, added to the slabs.  The stream orders the launches: a rectangle is consumed
+// before the next one overwrites the ring.
+static int tc_adjoint_chunked(const lory_dims& D, const WsPtrs& q, const bf16* x, const bf16* w1, const bf16* w2,
+                              const bf16* w3, const bf16* dy, bf16* dw1, bf16* dw2, bf16* dw3, cudaStream_t st) {
+  const int S = D.B * (D.L / D.T), T = D.T, d = D.d, f = D.f;
+  const AdjChunks ch = adjoint_chunks(D);
+  bf16* ring = q.dwbar1;
+  // matrix k: rows come from the columns of a_src (inner extent R[k]), columns from those of b_src (inner extent C[k])
+  const int R[3] = {f, f, d}, C[3] = {d, d, f};
+  const bf16* a_src[3] = {q.dG, q.dU, dy};
+  const bf16* b_src[3] = {x, x, q.H};
+  const bf16* wk[3] = {w1, w3, w2};
+  bf16* dwk[3] = {dw1, dw3, dw2};
+  LORY_CUDA_OK(cudaMemsetAsync(q.dw_partial, 0, (size_t)tc_dw_slabs(D) * S * D.E * sizeof(float), st));
+  for (int k = 0; k < 3; ++k) {
+    for (int r0 = 0; r0 < R[k]; r0 += ch.rows) {
+      for (int c0 = 0; c0 < C[k]; c0 += ch.cols[k]) {
+        const int Rc = R[k] - r0 < ch.rows ? R[k] - r0 : ch.rows;
+        const int Cc = C[k] - c0 < ch.cols[k] ? C[k] - c0 : ch.cols[k];
+        CUtensorMap m_a, m_b, m_o;
+        LORY_TRY(make_map(&m_a, a_src[k] + r0, Rc, T, S, R[k], (uint64_t)T * R[k], 64));
+        LORY_TRY(make_map(&m_b, b_src[k] + c0, Cc, T, S, C[k], (uint64_t)T * C[k], 64));
+        LORY_TRY(make_blocked_map(&m_o, ring, Rc, Cc, S, 64, 1, 1, 2));
+        TcGemmParams p = {};
+        p.groups = S; p.K = T; p.M = Rc; p.N = Cc; p.status = q.status;
+        if (R[k] >= 256)
+          LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true, 2>("wgrad", m_a, m_a, m_b, m_b, m_o,
+                                                                                      m_o, m_o, p, st)));
+        else
+          LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true>("wgrad", m_a, m_a, m_b, m_b, m_o, m_o,
+                                                                                   m_o, p, st)));
+        AdjPiece pc[3] = {};
+        const uint64_t off = (uint64_t)r0 * C[k] + c0;
+        pc[k] = AdjPiece{ring, wk[k] + off, dwk[k] + off, Rc, Cc, (uint64_t)f * d, (uint64_t)C[k]};
+        LORY_TRY(launch_stage2(D, q, pc, true, st));
+      }
+    }
+  }
+  return LORY_OK;
+}
+
 int tc_ffn_backward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* x, const bf16* w1, const bf16* w2,
                     const bf16* w3, const bf16* dy, bf16* dw1, bf16* dw2, bf16* dw3, cudaStream_t st) {
   const int S = D.B * (D.L / D.T), T = D.T, d = D.d, f = D.f;
@@ -483,6 +599,7 @@ int tc_ffn_backward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* 
       LORY_TRY((launch_tc<false, true, 256, MODE_PLAIN, EPI_DSWIGLU, true>("dh_dswiglu", m_dy, m_dy, m_b2, m_b2, m_dgo,
                                                                             m_duo, m_duo, p, st, &m_gi, &m_ui)));
   }
+  if (D.flags & LORY_FLAG_CHUNKED_ADJOINT) return tc_adjoint_chunked(D, q, x, w1, w2, w3, dy, dw1, dw2, dw3, st);
   // dWbar2[d, f] = dY^T H;  dWbar1[f, d] = dG^T X;  dWbar3[f, d] = dU^T X     (K = T), stored blocked
   {
     CUtensorMap m_dyT, m_h, m_dg, m_du, m_x, m_o2, m_o1, m_o3;
@@ -519,10 +636,10 @@ int tc_ffn_backward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* 
   }
   // adjoint of the merge
   {
-    const bf16* dsrc[3] = {q.dwbar1, q.dwbar3, q.dwbar2};
-    const bf16* wsrc[3] = {w1, w3, w2};
-    bf16* ddst[3] = {dw1, dw3, dw2};
-    LORY_TRY(launch_stage2(D, q, dsrc, wsrc, ddst, st));
+    const AdjPiece pc[3] = {{q.dwbar1, w1, dw1, f, d, (uint64_t)f * d, (uint64_t)d},
+                            {q.dwbar3, w3, dw3, f, d, (uint64_t)f * d, (uint64_t)d},
+                            {q.dwbar2, w2, dw2, d, f, (uint64_t)f * d, (uint64_t)f}};
+    LORY_TRY(launch_stage2(D, q, pc, false, st));
   }
   return LORY_OK;
 }

@@ -11,6 +11,9 @@ size_t tc_w_split_bytes(const lory_dims& D);
 bool tc_supported(const lory_dims& D);
 // Elements of the blocked layout of a per-segment [R, C] matrix over all segments.
 size_t tc_blocked_elems(const lory_dims& D, int R, int C);
+// Elements of the buffer the chunked adjoint (LORY_FLAG_CHUNKED_ADJOINT) keeps one rectangle of per-segment weight
+// gradients in: sized from the device's L2 (environment variable LORY_ADJOINT_CHUNK_MB overrides the budget).
+size_t tc_adjoint_ring_elems(const lory_dims& D);
 // Number of [S,E] partial slabs the tensor-core dw contraction writes.
 int tc_dw_slabs(const lory_dims& D);
 
