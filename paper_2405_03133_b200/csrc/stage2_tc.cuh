@@ -12,7 +12,12 @@
 // hi-weighted sums in accumulator rows 0..63 and lo-weighted sums in rows 64..127; the epilogue adds
 // the two halves.  With E <= 32 one 64-wide table holds hi in columns 0..31 and lo in 32..63 and is placed
 // in shared memory twice, so that all four epilogue warps have work: two per 64-column half of the tile.  The dw accumulator stays in TMEM for the whole kernel.
-// Roles as in the grouped GEMM: warp 0 TMA, warp 1 MMA, warps 2..5 epilogue.
+// Roles: warp 0 TMA, warp 1 issues the first product and owns TMEM, warps 2..5 epilogue, warp 6 issues the second
+// product.  Two issuing threads because with few segments a tile is small (24 KB at S = 64) and the instruction
+// stream of ONE thread issuing both products (12 MMAs with their descriptors, 2 commits, 2 waits) was what a tile
+// waited for (E = 8, S = 128: 0.51 -> 0.44 ms; E = 16, S = 64, d = 2048: 1.83 -> 1.65 ms); each stage is handed back
+// once both threads' MMAs have read it (its barrier counts two arrivals).  A third issuer (the second product split
+// by column block into accumulators of their own) measured no faster.
 #pragma once
 #include <cuda.h>
 
@@ -51,7 +56,7 @@ struct Stage2Params {
 
 // ACC: add the values already in the output tensors (gradient accumulation).
 template <bool ACC>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(224, 1)
 stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -94,7 +99,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < 8; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
-      ptx::mbar_init(&empty_bar[s], 1);
+      ptx::mbar_init(&empty_bar[s], 2);   // the two MMA-issuing threads
     }
     for (int a = 0; a < NACC; ++a) {
       ptx::mbar_init(&tmem_full_bar[a], 1);
@@ -168,7 +173,6 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc1 = ptx::make_idesc_bf16(128, 128, true, true);
-      const uint32_t idesc2 = ptx::make_idesc_bf16(128, p.Epad16, false, false);
       if (!ptx::mbar_wait(&w_bar, 0, &abort_flag)) {
         atomicOr(p.status, STATUS_TIMEOUT_MMA);
         abort_flag = 1;
@@ -178,24 +182,20 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
       // built once and the address added per instruction, which keeps this one thread's work per tile small.
       const uint64_t d1a = ptx::make_smem_desc(0, 16384, 1024);                    // w tile, lo 16 KB behind hi
       const uint64_t d1b = ptx::make_smem_desc(0, (uint32_t)p.cb_stride, 1024);    // dWbar tile as [segment, column]
-      const uint64_t d2ab = ptx::make_smem_desc(0, 16, 1024);                      // K-major tiles of the second product
-      const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4, cb16 = (uint32_t)p.cb_stride >> 4;
-      const uint32_t t16 = (uint32_t)(p.Epad16 * 128) >> 4;
+      const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
       const uint32_t stage0_16 = ptx::smem_u32(s_stage) >> 4, w16 = wbase >> 4;
       int s = 0;
-      uint32_t ph = 0, tcount = 0;
+      uint32_t ph = 0;
       uint32_t acc = 0, acc_ph = 0;   // accumulator ring position and phase
       for (int tile = blockIdx.x; tile < num_tiles;
-           tile += gridDim.x, ++tcount, acc = (acc + 1 == NACC ? 0 : acc + 1), acc_ph ^= (acc == 0)) {
+           tile += gridDim.x, acc = (acc + 1 == NACC ? 0 : acc + 1), acc_ph ^= (acc == 0)) {
         if (!ptx::mbar_wait(&tmem_empty_bar[acc], acc_ph ^ 1, &abort_flag)) {
           atomicOr(p.status, STATUS_TIMEOUT_MMA);
           abort_flag = 1;
         }
         const uint32_t tmem_d1 = tmem_base + acc * 128;
-        // debug build: both accumulators (the per-tile one and the resident dw one) inside the 512 columns
-        const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d1, tmem_base, 512, 128) &&
-                                           dbg::tmem_ok(tmem_d2, tmem_base, 512, (uint32_t)(p.s_tiles * p.Epad16)),
-                                       p.status);
+        // debug build: the per-tile accumulator inside the 512 columns
+        const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d1, tmem_base, 512, 128), p.status);
         for (int st = 0; st < p.s_tiles; ++st, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0)) {
           if (!ptx::mbar_wait(&full_bar[s], ph, &abort_flag)) {
             atomicOr(p.status, STATUS_TIMEOUT_MMA);
@@ -203,7 +203,6 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           }
           ptx::tc_fence_after_sync();
           const uint32_t d16 = stage0_16 + (uint32_t)s * stage16;   // this stage's dWbar tile, 16-byte units
-          const uint32_t tb16 = d16 + 2 * cb16;                     // its expert tile
           const uint32_t whi16 = w16 + (uint32_t)st * (32768u >> 4);
           const int rows = min(128, p.S - st * 128);
           const int ksteps = (rows + 15) / 16;
@@ -213,9 +212,33 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
             ptx::umma_bf16(tmem_d1, d1a | (uint64_t)(whi16 + kk * 128), d1b | (uint64_t)(d16 + kk * 128), idesc1,
                            (st > 0 || kk > 0) ? 1u : 0u);
           }
-          // dw [s, e] += dWbar [s, p] . W^T [p, e]   (one accumulator per group of 128 segments; with fewer than
-          // 128 segments in the box the rows past them hold whatever follows in shared memory, and their
-          // accumulator rows are never read)
+          ptx::umma_commit(&empty_bar[s]);
+        }
+        ptx::umma_commit(&tmem_full_bar[acc]);
+      }
+    }
+  } else if (warp == 6) {
+    // second product: dw [s, e] += dWbar [s, p] . W^T [p, e]   (one accumulator per group of 128 segments, resident
+    // in TMEM for the whole kernel; with fewer than 128 segments in the box the rows past them hold whatever follows
+    // in shared memory, and their accumulator rows are never read)
+    if (lane == 0) {
+      const uint32_t idesc2 = ptx::make_idesc_bf16(128, p.Epad16, false, false);
+      const uint64_t d2ab = ptx::make_smem_desc(0, 16, 1024);   // K-major tiles; only the 14-bit address varies
+      const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4, cb16 = (uint32_t)p.cb_stride >> 4;
+      const uint32_t t16 = (uint32_t)(p.Epad16 * 128) >> 4;
+      const uint32_t stage0_16 = ptx::smem_u32(s_stage) >> 4;
+      const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d2, tmem_base, 512, (uint32_t)(p.s_tiles * p.Epad16)), p.status);
+      int s = 0;
+      uint32_t ph = 0, tcount = 0;
+      for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tcount) {
+        for (int st = 0; st < p.s_tiles; ++st, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0)) {
+          if (!ptx::mbar_wait(&full_bar[s], ph, &abort_flag)) {
+            atomicOr(p.status, STATUS_TIMEOUT_MMA);
+            abort_flag = 1;
+          }
+          ptx::tc_fence_after_sync();
+          const uint32_t d16 = stage0_16 + (uint32_t)s * stage16;   // this stage's dWbar tile, 16-byte units
+          const uint32_t tb16 = d16 + 2 * cb16;                     // its expert tile
           const uint32_t tmem_d2s = tmem_d2 + st * p.Epad16;
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
@@ -229,7 +252,6 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           }
           ptx::umma_commit(&empty_bar[s]);
         }
-        ptx::umma_commit(&tmem_full_bar[acc]);
       }
       ptx::umma_commit(&d2_bar);
     }

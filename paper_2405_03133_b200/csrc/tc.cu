@@ -19,6 +19,7 @@
 #include "gemm_tc.cuh"
 #include "merge_tc.cuh"
 #include "stage2_tc.cuh"
+#include "wgrad_tc.cuh"
 
 namespace lory {
 
@@ -178,6 +179,49 @@ static int launch_tc(const char* label, const CUtensorMap& a0, const CUtensorMap
   }
   LORY_AFTER_LAUNCH();
   return LORY_OK;
+}
+
+// One per-segment weight gradient C_g = A_g^T B_g (K = T): the resident-operand kernel for CTA-pair tiles with short
+// segments (its strips run along the dimension with more tiles), else the grouped GEMM.  Measured on one GPU
+// (d = 2048, f = 5504, E = 32; three launches): T = 64: 3.69 -> 3.53 ms, T = 128: 1.99 -> 1.82 ms; at T = 256 the two
+// kernels tie (d = 1024, f = 2752: 0.591 vs 0.600 ms; d = 2048: 1.14 vs 1.11 ms) and the grouped GEMM stays.
+static int launch_wgrad(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, int M, int N, int K, int groups,
+                        bool pairs, uint32_t* status, cudaStream_t st) {
+  if (pairs && K <= 128) {
+    WgradParams p = {};
+    p.M = M; p.N = N; p.K = K; p.groups = groups; p.status = status;
+    p.m_tiles = (int)ceil_div(M, 256);
+    p.n_tiles = (int)ceil_div(N, 256);
+    const bool res_a = p.n_tiles >= p.m_tiles;
+    const long strips = (long)(res_a ? p.m_tiles : p.n_tiles) * groups;
+    if (strips <= 0) return LORY_OK;
+    if (strips > 0x7fffffffL) return LORY_ERR_SHAPE;
+    static bool attr_set[2][kMaxDevices];
+    LORY_TRY(allow_dynamic_smem(wgrad_kernel<false>, WgradTile::SMEM_BYTES, attr_set[0]));
+    LORY_TRY(allow_dynamic_smem(wgrad_kernel<true>, WgradTile::SMEM_BYTES, attr_set[1]));
+    const int slots = sm_count() / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (unsigned)(strips < slots ? strips : slots));
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = WgradTile::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    ProfScope ps("wgrad", st);
+    if (res_a) LORY_CUDA_OK(cudaLaunchKernelEx(&cfg, wgrad_kernel<true>, a, b, c, p));
+    else LORY_CUDA_OK(cudaLaunchKernelEx(&cfg, wgrad_kernel<false>, a, b, c, p));
+    LORY_AFTER_LAUNCH();
+    return LORY_OK;
+  }
+  TcGemmParams p = {};
+  p.groups = groups; p.K = K; p.M = M; p.N = N; p.status = status;
+  if (pairs) return launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true, 2>("wgrad", a, a, b, b, c, c, c, p, st);
+  return launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true>("wgrad", a, a, b, b, c, c, c, p, st);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -441,8 +485,8 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[
     p.S = S - base < 256 ? S - base : 256;
     p.s_tiles = (p.S + 127) / 128;
     ProfScope ps("stage2", st);
-    if (base > 0 || (D.flags & LORY_FLAG_ACCUMULATE_GRADS)) stage2_kernel<true><<<grid, 192, smem, st>>>(maps, p);
-    else stage2_kernel<false><<<grid, 192, smem, st>>>(maps, p);
+    if (base > 0 || (D.flags & LORY_FLAG_ACCUMULATE_GRADS)) stage2_kernel<true><<<grid, 224, smem, st>>>(maps, p);
+    else stage2_kernel<false><<<grid, 224, smem, st>>>(maps, p);
     LORY_AFTER_LAUNCH();
   }
   return LORY_OK;
@@ -555,14 +599,7 @@ static int tc_adjoint_chunked(const lory_dims& D, const WsPtrs& q, const bf16* x
         LORY_TRY(make_map(&m_a, a_src[k] + r0, Rc, T, S, R[k], (uint64_t)T * R[k], 64));
         LORY_TRY(make_map(&m_b, b_src[k] + c0, Cc, T, S, C[k], (uint64_t)T * C[k], 64));
         LORY_TRY(make_blocked_map(&m_o, ring, Rc, Cc, S, 64, 1, 1, 2));
-        TcGemmParams p = {};
-        p.groups = S; p.K = T; p.M = Rc; p.N = Cc; p.status = q.status;
-        if (R[k] >= 256)
-          LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true, 2>("wgrad", m_a, m_a, m_b, m_b, m_o,
-                                                                                      m_o, m_o, p, st)));
-        else
-          LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true>("wgrad", m_a, m_a, m_b, m_b, m_o, m_o,
-                                                                                   m_o, p, st)));
+        LORY_TRY(launch_wgrad(m_a, m_b, m_o, Rc, Cc, T, S, R[k] >= 256, q.status, st));
         AdjPiece pc[3] = {};
         const uint64_t off = (uint64_t)r0 * C[k] + c0;
         pc[k] = AdjPiece{ring, wk[k] + off, dwk[k] + off, Rc, Cc, (uint64_t)f * d, (uint64_t)C[k]};
@@ -611,28 +648,10 @@ int tc_ffn_backward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* 
     LORY_TRY(make_blocked_map(&m_o2, q.dwbar2, d, f, S, 64, 1, 1, 2));  // 128 rows x 64 cols per store
     LORY_TRY(make_blocked_map(&m_o1, q.dwbar1, f, d, S, 64, 1, 1, 2));
     LORY_TRY(make_blocked_map(&m_o3, q.dwbar3, f, d, S, 64, 1, 1, 2));
-    TcGemmParams p = {};
-    p.groups = S; p.K = T; p.status = q.status;
     // 256-row CTA-pair tiles whenever the output has at least 256 rows
-    p.M = d; p.N = f;
-    if (d >= 256)
-      LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true, 2>("wgrad", m_dyT, m_dyT, m_h, m_h, m_o2,
-                                                                                  m_o2, m_o2, p, st)));
-    else
-      LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true>("wgrad", m_dyT, m_dyT, m_h, m_h, m_o2,
-                                                                               m_o2, m_o2, p, st)));
-    p.M = f; p.N = d;
-    if (f >= 256) {
-      LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true, 2>("wgrad", m_dg, m_dg, m_x, m_x, m_o1,
-                                                                                  m_o1, m_o1, p, st)));
-      LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true, 2>("wgrad", m_du, m_du, m_x, m_x, m_o3,
-                                                                                  m_o3, m_o3, p, st)));
-    } else {
-      LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true>("wgrad", m_dg, m_dg, m_x, m_x, m_o1, m_o1,
-                                                                               m_o1, p, st)));
-      LORY_TRY((launch_tc<true, true, 256, MODE_PLAIN, EPI_BF16, false, true>("wgrad", m_du, m_du, m_x, m_x, m_o3, m_o3,
-                                                                               m_o3, p, st)));
-    }
+    LORY_TRY(launch_wgrad(m_dyT, m_h, m_o2, d, f, T, S, d >= 256, q.status, st));
+    LORY_TRY(launch_wgrad(m_dg, m_x, m_o1, f, d, T, S, f >= 256, q.status, st));
+    LORY_TRY(launch_wgrad(m_du, m_x, m_o3, f, d, T, S, f >= 256, q.status, st));
   }
   // adjoint of the merge
   {

@@ -95,6 +95,12 @@ TC_SMALL = [
     Workload("tc_T100", B=2, L=300, T=100, d=64, f=72, E=4, w_r_std=1.0),
     Workload("tc_T24_T_smaller_than_a_k_block", B=3, L=96, T=24, d=136, f=64, E=6, w_r_std=1.0),
     Workload("tc_T1", B=2, L=6, T=1, d=64, f=64, E=3, w_r_std=1.0),
+    # weight-gradient kernel with a resident operand (CTA-pair tiles, T <= 128): contraction tails (T = 100: two token
+    # blocks, the second ragged; T = 24: one), a second row tile that is almost empty (d = 264), and enough segments
+    # that every CTA pair takes several strips and both resident buffers change phase (400 segments, 74 pairs)
+    Workload("tc_wgrad_resident_T100", B=2, L=300, T=100, d=256, f=328, E=4, w_r_std=1.0),
+    Workload("tc_wgrad_resident_T24", B=3, L=96, T=24, d=264, f=256, E=6, w_r_std=1.0),
+    Workload("tc_wgrad_resident_400_segments", B=25, L=512, T=32, d=256, f=328, E=4, w_r_std=1.0),
     Workload("tc_288_segments", B=9, L=1024, T=32, d=64, f=72, E=4, w_r_std=1.0),
     Workload("tc_520_segments_40_experts", B=13, L=640, T=16, d=64, f=72, E=40, w_r_std=1.0),
 ]
