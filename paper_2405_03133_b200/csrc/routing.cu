@@ -104,11 +104,13 @@ __device__ __forceinline__ void write_weight_row(const float* p_sm, size_t row, 
     }
   }
   if (ex.comb) {
-    for (int c = lane; c < 64; c += 32) {
-      const int e = c & 31;
+    // [hi | lo | hi | hi | lo | lo], 32 columns each
+    for (int c = lane; c < 192; c += 32) {
+      const int e = c & 31, part = c >> 5;
       const float v = e < E ? p_sm[e] : 0.f;
       const bf16 h = __float2bfloat16_rn(v);
-      ex.comb[row * 64 + c] = c < 32 ? h : __float2bfloat16_rn(v - __bfloat162float(h));
+      const bool is_hi = part == 0 || part == 2 || part == 3;
+      ex.comb[row * 192 + c] = is_hi ? h : __float2bfloat16_rn(v - __bfloat162float(h));
     }
   }
 }

@@ -9,7 +9,7 @@ namespace lory {
 // prefix != 0: prefix routing (every segment of a sequence uses its first segment's p).
 // Optional extra outputs of the routing step, written by the router kernel itself:
 // a second copy of the routing weights (the caller's route_w), and the bf16 hi + lo tables of the weights that
-// the tensor-core merge reads: hi, lo [S, Epad]; comb [S, 64] = hi in columns 0..31, lo in 32..63 (E <= 32 only).
+// the tensor-core merge reads: hi, lo [S, Epad]; comb [S, 192] = [hi | lo | hi | hi | lo | lo] in groups of 32 columns (E <= 32 only).
 struct RouteExtra {
   float* w_copy = nullptr;
   bf16* hi = nullptr;

@@ -12,6 +12,11 @@
 // hi-weighted sums in accumulator rows 0..63 and lo-weighted sums in rows 64..127; the epilogue adds
 // the two halves.  With E <= 32 one 64-wide table holds hi in columns 0..31 and lo in 32..63 and is placed
 // in shared memory twice, so that all four epilogue warps have work: two per 64-column half of the tile.  The dw accumulator stays in TMEM for the whole kernel.
+// With E <= 32 and at most 64 segments (p.fast) the first product runs as two MMAs per 16 segments, [hi|hi] and
+// [lo|lo] tables into ONE accumulator: every 32-lane quarter then holds the finished sums of all experts, and the
+// epilogue warps take whole tiles in turn (two per accumulator, one 64-column half each) without exchanging
+// anything (d = 2048, f = 5504: E = 32, S = 16: 1.52 -> 1.17 ms; S = 64: 1.95 -> 1.64 ms; E = 16, S = 64: 1.65 -> 1.54 ms;
+// at S = 128 the doubled MMA count costs more than it saves, so the arrangement above stays there).
 // Roles: warp 0 TMA, warp 1 issues the first product and owns TMEM, warps 2..5 epilogue, warp 6 issues the second
 // product.  Two issuing threads because with few segments a tile is small (24 KB at S = 64) and the instruction
 // stream of ONE thread issuing both products (12 MMAs with their descriptors, 2 commits, 2 waits) was what a tile
@@ -42,7 +47,9 @@ struct Stage2Params {
   uint32_t cmagic[3];  // ceil(2^32 / ctiles), 0 for ctiles == 1: n / ctiles == __umulhi(n, cmagic) for every tile index n
   int tile_end[3];  // exclusive prefix sums of (rows rounded up to 64) * ctiles
   int cb_stride;    // bytes between the two 64-column blocks of a dWbar tile in shared memory (= segments per box * 128)
-  int dup;          // E <= 32: w_hi and w_lo are both the combined [hi (32) | lo (32)] table
+  int dup;          // E <= 32: w_hi and w_lo are both the combined table [hi | lo | hi | hi | lo | lo] (32 columns each)
+  int fast;         // E <= 32 and S <= 64: hi and lo sums meet in the accumulator (see the kernel)
+  int w_bytes;      // shared memory of the resident weight tiles
   int xch_bytes;    // one exchange buffer: 32 lanes x 256 B, or x 128 B with E <= 32
   int stages;       // pipeline depth (<= 8)
   int stage_bytes, tx_bytes;
@@ -60,9 +67,10 @@ __global__ void __launch_bounds__(224, 1)
 stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* s_w = smem;                                // [s_tiles][hi 16 KB | lo 16 KB]
-  uint8_t* s_out = smem + (size_t)p.s_tiles * 32768;  // 2 storing warps x 2 x 4 KB output staging
+  uint8_t* s_w = smem;                                // [s_tiles][hi 16 KB | lo 16 KB]; fast: [hi|hi, hi|hi, lo|lo, lo|lo] 16 KB each
+  uint8_t* s_out = smem + (size_t)p.w_bytes;          // 2 storing warps x 2 x 4 KB output staging
   uint8_t* s_xch = s_out + 16384;                     // 2 warp couples x 2 buffers: lo halves on their way to the hi warps
+                                                      // (fast: staging of the other two storing warps)
   uint8_t* s_stage = s_xch + 4 * p.xch_bytes;
   __shared__ __align__(8) uint64_t full_bar[8];
   __shared__ __align__(8) uint64_t empty_bar[8];
@@ -103,7 +111,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
     }
     for (int a = 0; a < NACC; ++a) {
       ptx::mbar_init(&tmem_full_bar[a], 1);
-      ptx::mbar_init(&tmem_empty_bar[a], 128);
+      ptx::mbar_init(&tmem_empty_bar[a], p.fast ? 64 : 128);   // fast: two warps read an accumulator
     }
     ptx::mbar_init(&w_bar, 1);
     ptx::mbar_init(&d2_bar, 1);
@@ -127,10 +135,19 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   if (warp == 0) {
     if (lane == 0) {
       // routing weights, once
-      ptx::mbar_expect_tx(&w_bar, (uint32_t)p.s_tiles * 32768u);
-      for (int st = 0; st < p.s_tiles; ++st) {
-        ptx::tma_load_3d(s_w + st * 32768, &maps.w_hi, &w_bar, 0, p.seg_base + st * 128, 0);
-        ptx::tma_load_3d(s_w + st * 32768 + 16384, &maps.w_lo, &w_bar, 0, p.seg_base + st * 128, 0);
+      ptx::mbar_expect_tx(&w_bar, p.fast ? 65536u : (uint32_t)p.s_tiles * 32768u);
+      if (p.fast) {
+        // columns 64..127 of the combined table are [hi | hi], 128..191 [lo | lo]; each tile sits in shared memory
+        // twice, so that the MMA's second 64-row group repeats the first
+        for (int h = 0; h < 2; ++h) {
+          ptx::tma_load_3d(s_w + h * 16384, &maps.w_hi, &w_bar, 64, p.seg_base, 0);
+          ptx::tma_load_3d(s_w + 32768 + h * 16384, &maps.w_hi, &w_bar, 128, p.seg_base, 0);
+        }
+      } else {
+        for (int st = 0; st < p.s_tiles; ++st) {
+          ptx::tma_load_3d(s_w + st * 32768, &maps.w_hi, &w_bar, 0, p.seg_base + st * 128, 0);
+          ptx::tma_load_3d(s_w + st * 32768 + 16384, &maps.w_lo, &w_bar, 0, p.seg_base + st * 128, 0);
+        }
       }
       uint32_t issued = 0, last_parity = 0;
       int s = 0;          // position in the stage ring and its phase, advanced by hand: a division per tile on
@@ -208,9 +225,18 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           const int ksteps = (rows + 15) / 16;
           // rows 0..63: w_hi^T [e, s] . dWbar [s, p]; rows 64..127: w_lo^T . dWbar (the A operand's second
           // 64-row group lies 16 KB after the first: that is the lo tile)
-          for (int kk = 0; kk < ksteps && acc_ok; ++kk) {
-            ptx::umma_bf16(tmem_d1, d1a | (uint64_t)(whi16 + kk * 128), d1b | (uint64_t)(d16 + kk * 128), idesc1,
-                           (st > 0 || kk > 0) ? 1u : 0u);
+          if (p.fast) {
+            // every 32-row quarter: (w_hi + w_lo)^T [e, s] . dWbar [s, p], the two halves as two MMAs into one accumulator
+            for (int kk = 0; kk < ksteps && acc_ok; ++kk) {
+              const uint64_t bdesc = d1b | (uint64_t)(d16 + kk * 128);
+              ptx::umma_bf16(tmem_d1, d1a | (uint64_t)(w16 + kk * 128), bdesc, idesc1, kk > 0 ? 1u : 0u);
+              ptx::umma_bf16(tmem_d1, d1a | (uint64_t)(w16 + (32768u >> 4) + kk * 128), bdesc, idesc1, 1u);
+            }
+          } else {
+            for (int kk = 0; kk < ksteps && acc_ok; ++kk) {
+              ptx::umma_bf16(tmem_d1, d1a | (uint64_t)(whi16 + kk * 128), d1b | (uint64_t)(d16 + kk * 128), idesc1,
+                             (st > 0 || kk > 0) ? 1u : 0u);
+            }
           }
           ptx::umma_commit(&empty_bar[s]);
         }
@@ -274,9 +300,65 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
     // this lane's bf16 row (128 values, or 64 with E <= 32), its 16-byte chunks swizzled by lane
     const int xlane = p.xch_bytes >> 5, xmask = (xlane >> 4) - 1;
     uint8_t* xch = s_xch + pair * 2 * p.xch_bytes + lane * xlane;
+    if (p.fast) {
+      // Every 32-lane quarter of an accumulator holds the finished sums of all (<= 32) experts.  Warps 0, 1 of this
+      // role take the tiles of accumulator 0 (this CTA's even tiles), warps 2, 3 those of accumulator 1, one 64-column
+      // half each: no exchange between warps, and a warp has two tile periods for its load - convert - store chain.
+      const int my_acc = q >> 1, half = q & 1;
+      wsg.buf = s_out + q * 8192;   // four storing warps: the exchange buffers serve as staging too
+      uint32_t n = 0;
+      for (int tile = blockIdx.x + my_acc * gridDim.x; tile < num_tiles; tile += 2 * gridDim.x, ++n) {
+        int k, row, c0;
+        decode(tile, k, row, c0);
+        if (!ptx::mbar_wait(&tmem_full_bar[my_acc], n & 1u, &abort_flag)) {
+          atomicOr(p.status, STATUS_TIMEOUT_EPI);
+          abort_flag = 1;
+        }
+        __syncwarp();  // every lane polls by itself; the warp-wide tcgen05 instructions below need it whole again
+        ptx::tc_fence_after_sync();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + my_acc * 128 + half * 64;
+        if (!dbg::check(tile_ok(k, row, c0) && dbg::tmem_ok(taddr, tmem_base, 512, 64) && dbg::smem_ok(wsg.buf, 8192),
+                        p.status)) {
+          ptx::tc_fence_before_sync();
+          ptx::mbar_arrive(&tmem_empty_bar[my_acc]);
+          continue;
+        }
+        uint32_t r[64];
+        ptx::tmem_ld_32x64(taddr, r);
+        const int col0 = c0 + half * half_col, rowc = row + half * half_row;
+        uint4 old[8];
+        if (ACC) {  // gradient accumulation: this lane's 64 old values (expert `lane`), zero where the tile leaves the tensor
+          const bool row_ok = lane < p.E && rowc < p.rows[k];
+          const __nv_bfloat16* src = p.acc_base[k] + (size_t)lane * p.e_stride[k] + (size_t)rowc * p.row_stride[k] + col0;
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            old[j] = (row_ok && col0 + 8 * j < p.cols[k]) ? *reinterpret_cast<const uint4*>(src + 8 * j)
+                                                          : make_uint4(0u, 0u, 0u, 0u);
+        }
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before_sync();
+        ptx::mbar_arrive(&tmem_empty_bar[my_acc]);   // the values are in registers: the accumulator may be reused
+        uint32_t w[32];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t ol[4] = {ACC ? old[j].x : 0u, ACC ? old[j].y : 0u, ACC ? old[j].z : 0u, ACC ? old[j].w : 0u};
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            float a = __uint_as_float(r[8 * j + 2 * t]), b = __uint_as_float(r[8 * j + 2 * t + 1]);
+            if (ACC) {
+              const float2 o2 = unpack_bf16(ol[t]);
+              a += o2.x;
+              b += o2.y;
+            }
+            w[4 * j + t] = pack_bf16(a, b);
+          }
+        }
+        warp_stage_and_store(wsg, &maps.out[k], col0, 0, rowc, lane, w);
+      }
+    }
     uint32_t it = 0;
     uint32_t acc = 0, acc_ph = 0;   // accumulator ring position and phase
-    for (int tile = blockIdx.x; tile < num_tiles;
+    for (int tile = p.fast ? num_tiles : (int)blockIdx.x; tile < num_tiles;
          tile += gridDim.x, ++it, acc = (acc + 1 == NACC ? 0 : acc + 1), acc_ph ^= (acc == 0)) {
       int k, row, c0;
       decode(tile, k, row, c0);

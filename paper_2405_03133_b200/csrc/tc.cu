@@ -230,11 +230,12 @@ static int launch_wgrad(const CUtensorMap& a, const CUtensorMap& b, const CUtens
 static int e_pad(const lory_dims& D) { return (D.E + 7) / 8 * 8; }
 static int e_pad16(const lory_dims& D) { return (D.E + 15) / 16 * 16; }
 
-// Routing weights as bf16 hi + lo tables [S, Epad].  With E <= 32 also one [S, 64] table `comb` with hi in
-// columns 0..31 and lo in columns 32..63 of each row (zero where e >= E); the grid then covers S x 64.
+// Routing weights as bf16 hi + lo tables [S, Epad].  With E <= 32 also one [S, 192] table `comb` holding, in groups
+// of 32 columns, [hi | lo | hi | hi | lo | lo] (zero where e >= E): the merge adjoint reads columns 0..63 or
+// 64..191 of it; the grid then covers S x 192.
 __global__ void split_w_kernel(const float* __restrict__ w, bf16* __restrict__ hi, bf16* __restrict__ lo,
                                bf16* __restrict__ comb, int S, int E, int Epad) {
-  const int width = E <= 32 ? 64 : Epad;
+  const int width = E <= 32 ? 192 : Epad;
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= S * width) return;
   const int s = i / width, c = i - s * width;
@@ -243,7 +244,8 @@ __global__ void split_w_kernel(const float* __restrict__ w, bf16* __restrict__ h
   const bf16 h = __float2bfloat16_rn(v);
   const bf16 l = __float2bfloat16_rn(v - __bfloat162float(h));
   if (E <= 32) {
-    comb[i] = c < 32 ? h : l;
+    const int part = c >> 5;
+    comb[i] = (part == 0 || part == 2 || part == 3) ? h : l;
     if (c >= Epad) return;
   }
   hi[(size_t)s * Epad + e] = h;
@@ -252,7 +254,7 @@ __global__ void split_w_kernel(const float* __restrict__ w, bf16* __restrict__ h
 
 size_t tc_w_split_bytes(const lory_dims& D) {
   const size_t S = (size_t)D.B * (D.L / D.T);
-  return 2 * align_up(S * e_pad(D) * 2, 256) + align_up(S * 64 * 2, 256);
+  return 2 * align_up(S * e_pad(D) * 2, 256) + align_up(S * 192 * 2, 256);
 }
 
 // The merge and merge-adjoint kernels keep the routing weights of the segments they work on resident in shared
@@ -446,8 +448,11 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[
   const uint32_t seg_box = S >= 128 ? 128u : (uint32_t)((S + 15) / 16 * 16);
   p.cb_stride = (int)seg_box * 128;
   p.dup = E <= 32 ? 1 : 0;
+  // E <= 32 and at most 64 segments: both weight halves go through the tensor core into the same accumulator,
+  // every 32-lane quarter of it holds the finished sums, and the epilogue warps take whole tiles in turn
+  p.fast = (p.dup && S <= 64) ? 1 : 0;
   if (p.dup) {
-    LORY_TRY(make_map(&maps.w_hi, q.w_comb, 64, S, 1, 64, 0, 128));
+    LORY_TRY(make_map(&maps.w_hi, q.w_comb, 192, S, 1, 192, 0, 128));
     maps.w_lo = maps.w_hi;
   } else {
     LORY_TRY(make_map(&maps.w_hi, q.w_hi, Ep, S, 1, Ep, 0, 128));
@@ -469,7 +474,8 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[
   p.xch_bytes = p.dup ? 4096 : 8192;
   // w tiles, output staging, lo/hi exchange; and, when the box has fewer than 128 segments, room behind the last
   // stage for the 128-row operand reads of the second product (rows past the box are read and never used)
-  const int fixed = p.s_tiles * 32768 + 16384 + 4 * p.xch_bytes + 1024 + (16384 - p.cb_stride);
+  p.w_bytes = p.fast ? 65536 : p.s_tiles * 32768;
+  const int fixed = p.w_bytes + 16384 + 4 * p.xch_bytes + 1024 + (16384 - p.cb_stride);
   p.stages = (kMaxSmem - fixed) / p.stage_bytes;
   if (p.stages > 8) p.stages = 8;
   if (p.stages < 2) return LORY_ERR_SHAPE;
@@ -508,7 +514,7 @@ int tc_ffn_forward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* x
   if (!(D.flags & LORY_FLAG_REUSE_MERGED)) {
     if (!w_is_split) {
       prof_begin("split_w", st);
-      split_w_kernel<<<(unsigned)ceil_div((long)S * (E <= 32 ? 64 : Ep), 256), 256, 0, st>>>(q.w, q.w_hi, q.w_lo, q.w_comb, S, E, Ep);
+      split_w_kernel<<<(unsigned)ceil_div((long)S * (E <= 32 ? 192 : Ep), 256), 256, 0, st>>>(q.w, q.w_hi, q.w_lo, q.w_comb, S, E, Ep);
       prof_end(st);
       LORY_AFTER_LAUNCH();
     }
