@@ -74,9 +74,12 @@ typedef enum { LORY_FP32 = 0, LORY_BF16 = 1 } lory_dtype;
                                         consumed from there, instead of being written out for the whole matrices.
                                         Same results up to the summation order of the routing gradient; the
                                         backward workspace shrinks by almost the size of the merged weights (2.1 GB
-                                        at E = 32, T = 256, d = 1024, f = 2752); about twice the launches of the
-                                        default backward and slower (measurements in the design notes).  Ignored
-                                        by the plain-FMA pipeline.  Pass it to lory_moe_workspace_bytes as well. */
+                                        at E = 32, T = 256, d = 1024, f = 2752); two launches per rectangle (68
+                                        instead of 4 there) and a slower step (3.5 against 2.7 ms), because this
+                                        GPU's L2 writes the buffer back to memory all the same.  Ignored by the
+                                        plain-FMA pipeline.  Pass it to lory_moe_workspace_bytes as well; the
+                                        buffer size follows the environment variable LORY_ADJOINT_CHUNK_MB (MiB)
+                                        when set, read by both calls. */
 
 /*
  * Problem description.  B sequences of L tokens, segment length T (L % T == 0),
