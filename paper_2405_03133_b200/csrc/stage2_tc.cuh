@@ -20,9 +20,12 @@
 // Roles: warp 0 TMA, warp 1 issues the first product and owns TMEM, warps 2..5 epilogue, warp 6 issues the second
 // product.  Two issuing threads because with few segments a tile is small (24 KB at S = 64) and the instruction
 // stream of ONE thread issuing both products (12 MMAs with their descriptors, 2 commits, 2 waits) was what a tile
-// waited for (E = 8, S = 128: 0.51 -> 0.44 ms; E = 16, S = 64, d = 2048: 1.83 -> 1.65 ms); each stage is handed back
+// waited for (E = 8, S = 128: 0.52 -> 0.45 ms; E = 16, S = 64, d = 2048: 1.83 -> 1.65 ms); each stage is handed back
 // once both threads' MMAs have read it (its barrier counts two arrivals).  A third issuer (the second product split
-// by column block into accumulators of their own) measured no faster.
+// by column block into accumulators of their own) measured no faster.  Where the kernel waits for memory anyway
+// (more than 64 segments and more than 16 experts: E = 32, S = 128) the second issuer measured 5 % SLOWER on the
+// same GPU (0.57 -> 0.60 ms, 12 % more DRAM reads: tiles that share fetched lines drift apart), so there warp 1
+// issues both products (p.split = 0) and warp 6 idles.
 #pragma once
 #include <cuda.h>
 
@@ -48,6 +51,7 @@ struct Stage2Params {
   int tile_end[3];  // exclusive prefix sums of (rows rounded up to 64) * ctiles
   int cb_stride;    // bytes between the two 64-column blocks of a dWbar tile in shared memory (= segments per box * 128)
   int dup;          // E <= 32: w_hi and w_lo are both the combined table [hi | lo | hi | hi | lo | lo] (32 columns each)
+  int split;        // the second product is issued by a warp of its own
   int fast;         // E <= 32 and S <= 64: hi and lo sums meet in the accumulator (see the kernel)
   int w_bytes;      // shared memory of the resident weight tiles
   int xch_bytes;    // one exchange buffer: 32 lanes x 256 B, or x 128 B with E <= 32
@@ -107,7 +111,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < 8; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
-      ptx::mbar_init(&empty_bar[s], 2);   // the two MMA-issuing threads
+      ptx::mbar_init(&empty_bar[s], p.split ? 2 : 1);   // one arrival per MMA-issuing thread
     }
     for (int a = 0; a < NACC; ++a) {
       ptx::mbar_init(&tmem_full_bar[a], 1);
@@ -131,6 +135,26 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_smem;
   const uint32_t tmem_d2 = tmem_base + NACC * 128;
+
+  // second product of one stage: dw [s, e] += dWbar [s, p] . W^T [p, e]   (one accumulator per group of 128 segments,
+  // resident in TMEM for the whole kernel; with fewer than 128 segments in the box the rows past them hold whatever
+  // follows in shared memory, and their accumulator rows are never read).  d16: the stage's address in 16-byte units.
+  const uint32_t idesc2 = ptx::make_idesc_bf16(128, p.Epad16, false, false);
+  auto issue_second = [&](uint32_t d16, int st, bool first) {
+    const uint64_t d2ab = ptx::make_smem_desc(0, 16, 1024);   // K-major tiles; only the 14-bit address varies
+    const uint32_t cb16 = (uint32_t)p.cb_stride >> 4, t16 = (uint32_t)(p.Epad16 * 128) >> 4;
+    const uint32_t tb16 = d16 + 2 * cb16;                     // the stage's expert tile
+    const uint32_t tmem_d2s = tmem_d2 + st * p.Epad16;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+#pragma unroll
+      for (int k16 = 0; k16 < 4; ++k16) {
+        const uint64_t adesc = d2ab | (uint64_t)(d16 + j * cb16 + k16 * 2);
+        const uint64_t bdesc = d2ab | (uint64_t)(tb16 + j * t16 + k16 * 2);
+        ptx::umma_bf16(tmem_d2s, adesc, bdesc, idesc2, (!first || j > 0 || k16 > 0) ? 1u : 0u);
+      }
+    }
+  };
 
   if (warp == 0) {
     if (lane == 0) {
@@ -202,10 +226,11 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
       const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
       const uint32_t stage0_16 = ptx::smem_u32(s_stage) >> 4, w16 = wbase >> 4;
       int s = 0;
-      uint32_t ph = 0;
+      uint32_t ph = 0, tcount = 0;
+      const bool d2_ok = dbg::check(dbg::tmem_ok(tmem_d2, tmem_base, 512, (uint32_t)(p.s_tiles * p.Epad16)), p.status);
       uint32_t acc = 0, acc_ph = 0;   // accumulator ring position and phase
       for (int tile = blockIdx.x; tile < num_tiles;
-           tile += gridDim.x, acc = (acc + 1 == NACC ? 0 : acc + 1), acc_ph ^= (acc == 0)) {
+           tile += gridDim.x, ++tcount, acc = (acc + 1 == NACC ? 0 : acc + 1), acc_ph ^= (acc == 0)) {
         if (!ptx::mbar_wait(&tmem_empty_bar[acc], acc_ph ^ 1, &abort_flag)) {
           atomicOr(p.status, STATUS_TIMEOUT_MMA);
           abort_flag = 1;
@@ -238,20 +263,17 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
                              (st > 0 || kk > 0) ? 1u : 0u);
             }
           }
+          if (!p.split && d2_ok) issue_second(d16, st, tcount == 0);   // no second issuer: both products from here
           ptx::umma_commit(&empty_bar[s]);
         }
         ptx::umma_commit(&tmem_full_bar[acc]);
       }
+      if (!p.split) ptx::umma_commit(&d2_bar);
     }
   } else if (warp == 6) {
-    // second product: dw [s, e] += dWbar [s, p] . W^T [p, e]   (one accumulator per group of 128 segments, resident
-    // in TMEM for the whole kernel; with fewer than 128 segments in the box the rows past them hold whatever follows
-    // in shared memory, and their accumulator rows are never read)
-    if (lane == 0) {
-      const uint32_t idesc2 = ptx::make_idesc_bf16(128, p.Epad16, false, false);
-      const uint64_t d2ab = ptx::make_smem_desc(0, 16, 1024);   // K-major tiles; only the 14-bit address varies
-      const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4, cb16 = (uint32_t)p.cb_stride >> 4;
-      const uint32_t t16 = (uint32_t)(p.Epad16 * 128) >> 4;
+    // the second product from a thread of its own (p.split)
+    if (lane == 0 && p.split) {
+      const uint32_t stage16 = (uint32_t)p.stage_bytes >> 4;
       const uint32_t stage0_16 = ptx::smem_u32(s_stage) >> 4;
       const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d2, tmem_base, 512, (uint32_t)(p.s_tiles * p.Epad16)), p.status);
       int s = 0;
@@ -263,19 +285,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
             abort_flag = 1;
           }
           ptx::tc_fence_after_sync();
-          const uint32_t d16 = stage0_16 + (uint32_t)s * stage16;   // this stage's dWbar tile, 16-byte units
-          const uint32_t tb16 = d16 + 2 * cb16;                     // its expert tile
-          const uint32_t tmem_d2s = tmem_d2 + st * p.Epad16;
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-#pragma unroll
-            for (int k16 = 0; k16 < 4; ++k16) {
-              if (!acc_ok) continue;
-              const uint64_t adesc = d2ab | (uint64_t)(d16 + j * cb16 + k16 * 2);
-              const uint64_t bdesc = d2ab | (uint64_t)(tb16 + j * t16 + k16 * 2);
-              ptx::umma_bf16(tmem_d2s, adesc, bdesc, idesc2, (tcount > 0 || j > 0 || k16 > 0) ? 1u : 0u);
-            }
-          }
+          if (acc_ok) issue_second(stage0_16 + (uint32_t)s * stage16, st, tcount == 0);
           ptx::umma_commit(&empty_bar[s]);
         }
       }

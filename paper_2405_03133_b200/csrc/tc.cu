@@ -451,6 +451,7 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[
   // E <= 32 and at most 64 segments: both weight halves go through the tensor core into the same accumulator,
   // every 32-lane quarter of it holds the finished sums, and the epilogue warps take whole tiles in turn
   p.fast = (p.dup && S <= 64) ? 1 : 0;
+  p.split = (S > 64 && E > 16) ? 0 : 1;   // measured: see the kernel's header
   if (p.dup) {
     LORY_TRY(make_map(&maps.w_hi, q.w_comb, 192, S, 1, 192, 0, 128));
     maps.w_lo = maps.w_hi;
