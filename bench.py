@@ -128,9 +128,9 @@ def implementation_bytes_per_step(wl):
 # the digest of the CUDA sources at that time, and a different digest turns the reported traffic into null.
 NCU_TRAFFIC = {
     "C3": {
-        "sources_sha1": "078a97370609eb6864e46f1de2c980afc6a0e5f9",
-        "bytes": {"pool_router": 68e6, "merge": 2747e6, "gemm1_swiglu": 2019e6, "gemm2": 965e6, "dh_dswiglu": 1488e6,
-                  "wgrad": 909e6, "stage2": 3394e6, "router_backward": 3e6, "dx": 1876e6},
+        "sources_sha1": "079d4bef069afda6255f129da43b6372d9be0476",
+        "bytes": {"pool_router": 68e6, "merge": 2753e6, "gemm1_swiglu": 2017e6, "gemm2": 965e6, "dh_dswiglu": 1486e6,
+                  "wgrad": 908e6, "stage2": 3229e6, "router_backward": 3e6, "dx": 1875e6},
     },
 }
 

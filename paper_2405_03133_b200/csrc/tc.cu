@@ -395,7 +395,7 @@ static int launch_merge(const lory_dims& D, const WsPtrs& q, const bf16* const s
   int acc = 0;
   for (int k = 0; k < 3; ++k) {
     LORY_TRY(make_expert_map(&maps.theta[k], src[k], R[k], C[k], E, p.Epad16));
-    LORY_TRY(make_blocked_map(&maps.out[k], dst[k], R[k], C[k], S, 1, 32, 1, 1));
+    LORY_TRY(make_blocked_map(&maps.out[k], dst[k], R[k], C[k], S, 1, S < 32 ? (uint32_t)S : 32u, 1, 1));  // no box rows past the segments
     p.ctiles[k] = (C[k] + (256 >> p.rpt_shift) - 1) / (256 >> p.rpt_shift);
     acc += (((R[k] + 63) / 64 * 64) >> p.rpt_shift) * p.ctiles[k];  // padded rows are written too (as zeros)
     p.tile_end[k] = acc;
