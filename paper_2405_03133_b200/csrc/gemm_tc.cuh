@@ -43,16 +43,22 @@ struct TcGemmParams {
 
 // CTAS = 2: two CTAs of a cluster share one 256 x BN tile (tcgen05 cta_group::2); each loads its own
 // 128 rows of A and one half of B's BN columns, which cuts the L2 -> shared-memory traffic per flop by a third.
-template <int BN, int EPI, int CTAS = 1>
+// AROWS < 128 (groups of at most AROWS rows: a decode step): only AROWS rows of A are loaded per stage, and the
+// shared memory that frees goes into more stages, i.e. more weight bytes in flight per SM.  The MMA still reads 128
+// rows; rows AROWS.. of its A operand are whatever follows in shared memory (inside the CTA's allocation: the output
+// staging follows the last stage), they only reach accumulator rows that are never stored.
+template <int BN, int EPI, int CTAS = 1, int AROWS = 128>
 struct TcTile {
   static constexpr int BM = 128, BK = 64;
-  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int A_BYTES = AROWS * BK * 2;
   static constexpr int B_BYTES = (BN / CTAS) * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  // the SwiGLU-backward epilogue trades pipeline stages for two input staging tiles (G, U)
-  static constexpr int STAGES = (CTAS == 2) ? ((EPI == EPI_DSWIGLU) ? 5 : 6)
-                                            : ((EPI == EPI_DSWIGLU) ? 3 : ((BN == 256) ? 4 : 6));
   static constexpr int OUT_BYTES = 128 * 128;  // one 128-row x 64-column bf16 staging tile
+  static constexpr int NARROW_STAGES = (227 * 1024 - 512 - 2 * OUT_BYTES - 1024) / STAGE_BYTES;
+  // the SwiGLU-backward epilogue trades pipeline stages for two input staging tiles (G, U)
+  static constexpr int STAGES = (AROWS < 128) ? (NARROW_STAGES > 16 ? 16 : NARROW_STAGES)
+                                : (CTAS == 2) ? ((EPI == EPI_DSWIGLU) ? 5 : 6)
+                                              : ((EPI == EPI_DSWIGLU) ? 3 : ((BN == 256) ? 4 : 6));
   static constexpr int IN_BYTES = (EPI == EPI_DSWIGLU) ? 2 * OUT_BYTES : 0;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_BYTES + IN_BYTES + 1024;  // + alignment slack
 };
@@ -137,14 +143,16 @@ __device__ __forceinline__ void warp_stage_and_store(WarpStager& ws, const CUten
   }
   ws.n++;
 }
-template <bool A_MN, bool B_MN, int BN, int MODE, int EPI, bool B_BLK = false, bool C_BLK = false, int CTAS = 1>
+template <bool A_MN, bool B_MN, int BN, int MODE, int EPI, bool B_BLK = false, bool C_BLK = false, int CTAS = 1,
+          int AROWS = 128>
 __global__ void __launch_bounds__(192, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
                const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                const __grid_constant__ CUtensorMap tmC2, const __grid_constant__ CUtensorMap tmE0,
                const __grid_constant__ CUtensorMap tmE1, const TcGemmParams p) {
-  using Tile = TcTile<BN, EPI, CTAS>;
+  using Tile = TcTile<BN, EPI, CTAS, AROWS>;
+  static_assert(AROWS == 128 || (!A_MN && CTAS == 1 && EPI != EPI_DSWIGLU), "short A tiles: K-major A, single CTA");
   constexpr bool PAIR = (CTAS == 2);
   const int rank = PAIR ? (int)ptx::cluster_ctarank() : 0;  // 0 = leader: arms the full barriers, issues the MMAs
   const int wid = blockIdx.x / CTAS, wstride = gridDim.x / CTAS;
@@ -202,7 +210,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      uint32_t it = 0;
+      int s = 0;        // position in the stage ring and its phase, advanced by hand (no division per stage)
+      uint32_t ph = 0;
       uint32_t issued = 0, last_parity = 0;
       bool ok = true;
       for (int tile = wid; tile < num_tiles; tile += wstride) {
@@ -223,9 +232,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           n0 = 0;
           gc = 0;
         }
-        for (int i = 0; i < total; ++i, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+        for (int i = 0; i < total; ++i, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0)) {
           if (!ptx::mbar_wait(&empty_bar[s], ph ^ 1, &abort_flag)) {
             atomicOr(p.status, STATUS_TIMEOUT_TMA);
             abort_flag = 1;
@@ -301,10 +308,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = ptx::make_idesc_bf16(128 * CTAS, BN, A_MN, B_MN);
-      uint32_t it = 0, tile_iter = 0;
+      // Shared-memory descriptors differ only in their 14-bit address field (16-byte units): the constant part is
+      // built once, the stage ring advances by hand, and per MMA only an addition is left (measured neutral for
+      // these GEMMs, whose MMAs are long; the merge adjoint, with its short ones, gained 10-16 % from the same).
+      const uint64_t adesc0 = A_MN ? ptx::make_smem_desc(0, 8192, 1024) : ptx::make_smem_desc(0, 16, 1024);
+      const uint64_t bdesc0 = B_MN ? ptx::make_smem_desc(0, 8192, 1024) : ptx::make_smem_desc(0, 16, 1024);
+      constexpr uint32_t a_step16 = (A_MN ? 2048u : 32u) >> 4, b_step16 = (B_MN ? 2048u : 32u) >> 4;
+      const uint32_t smem16 = ptx::smem_u32(smem) >> 4;
+      int s = 0;
+      uint32_t ph = 0, tile_iter = 0;
+      const int nkb = (p.K + 63) / 64;
+      const int total = (MODE == MODE_DUALK) ? 2 * nkb : nkb;
       for (int tile = wid; tile < num_tiles; tile += wstride, ++tile_iter) {
-        const int nkb = (p.K + 63) / 64;
-        const int total = (MODE == MODE_DUALK) ? 2 * nkb : nkb;
         const uint32_t acc = tile_iter & 1;
         if (!ptx::mbar_wait(&tmem_empty_bar[acc], ((tile_iter >> 1) & 1) ^ 1, &abort_flag)) {
           atomicOr(p.status, STATUS_TIMEOUT_MMA);
@@ -313,22 +328,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         ptx::tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + acc * BN;
         const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d, tmem_base, 2 * BN, BN), p.status);
-        for (int i = 0; i < total; ++i, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+        for (int i = 0; i < total; ++i, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0)) {
           if (!ptx::mbar_wait(&full_bar[s], ph, &abort_flag)) {
             atomicOr(p.status, STATUS_TIMEOUT_MMA);
             abort_flag = 1;
           }
           ptx::tc_fence_after_sync();
-          const uint32_t a_addr = ptx::smem_u32(smem + (size_t)s * Tile::STAGE_BYTES);
-          const uint32_t b_addr = a_addr + Tile::A_BYTES;
+          const uint32_t a16 = smem16 + (uint32_t)s * (Tile::STAGE_BYTES >> 4);   // this stage, 16-byte units
+          const uint32_t b16 = a16 + (Tile::A_BYTES >> 4);
 #pragma unroll
           for (int k16 = 0; k16 < 4; ++k16) {
-            const uint64_t adesc = A_MN ? ptx::make_smem_desc(a_addr + k16 * 2048, 8192, 1024)
-                                        : ptx::make_smem_desc(a_addr + k16 * 32, 16, 1024);
-            const uint64_t bdesc = B_MN ? ptx::make_smem_desc(b_addr + k16 * 2048, 8192, 1024)
-                                        : ptx::make_smem_desc(b_addr + k16 * 32, 16, 1024);
+            const uint64_t adesc = adesc0 | (uint64_t)((a16 + k16 * a_step16) & 0x3FFFu);
+            const uint64_t bdesc = bdesc0 | (uint64_t)((b16 + k16 * b_step16) & 0x3FFFu);
             if (!acc_ok) continue;  // debug build: an accumulator outside the TMEM allocation is never written
             if (PAIR) ptx::umma_bf16_pair(tmem_d, adesc, bdesc, idesc, (i > 0 || k16 > 0) ? 1u : 0u);
             else ptx::umma_bf16(tmem_d, adesc, bdesc, idesc, (i > 0 || k16 > 0) ? 1u : 0u);

@@ -140,19 +140,20 @@ static int allow_dynamic_smem(K kern, int bytes, bool (&done)[kMaxDevices]) {
 
 static const int kMaxSmem = 227 * 1024 - 512;  // dynamic shared memory we may ask for (static use is < 512 B)
 
-template <bool A_MN, bool B_MN, int BN, int MODE, int EPI, bool B_BLK = false, bool C_BLK = false, int CTAS = 1>
+template <bool A_MN, bool B_MN, int BN, int MODE, int EPI, bool B_BLK = false, bool C_BLK = false, int CTAS = 1,
+          int AROWS = 128>
 static int launch_tc(const char* label, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0,
                      const CUtensorMap& b1, const CUtensorMap& c0, const CUtensorMap& c1, const CUtensorMap& c2,
                      TcGemmParams p, cudaStream_t st, const CUtensorMap* e0 = nullptr,
                      const CUtensorMap* e1 = nullptr) {
   constexpr int TILE_N = (MODE == MODE_DUALB) ? BN / 2 : BN;
-  using Tile = TcTile<BN, EPI, CTAS>;
+  using Tile = TcTile<BN, EPI, CTAS, AROWS>;
   p.m_tiles = (int)ceil_div(p.M, 128 * CTAS);
   p.n_tiles = (int)ceil_div(p.N, TILE_N);
   const long tiles = (long)p.m_tiles * p.n_tiles * p.groups;
   if (tiles <= 0) return LORY_OK;
   if (tiles > 0x7fffffffL) return LORY_ERR_SHAPE;
-  auto kern = tc_gemm_kernel<A_MN, B_MN, BN, MODE, EPI, B_BLK, C_BLK, CTAS>;
+  auto kern = tc_gemm_kernel<A_MN, B_MN, BN, MODE, EPI, B_BLK, C_BLK, CTAS, AROWS>;
   static bool attr_set[kMaxDevices];
   LORY_TRY(allow_dynamic_smem(kern, Tile::SMEM_BYTES, attr_set));
   const int slots = sm_count() / CTAS;  // persistent CTAs (or CTA pairs)
@@ -536,7 +537,12 @@ int tc_ffn_forward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* x
     LORY_TRY(make_map(&m_h, q.H, f, T, S, f, (uint64_t)T * f, 32));
     TcGemmParams p = {};
     p.M = T; p.N = f; p.K = d; p.groups = S; p.status = q.status;
-    if (use_pairs(T))  // leader loads the Wbar1 rows (G half of the accumulator), its peer the Wbar3 rows (U half)
+    if (T <= 32) {  // a decode step: 32-row A tiles, the freed shared memory holds more weight stages
+      CUtensorMap m_xs;
+      LORY_TRY(make_map(&m_xs, x, d, T, S, d, (uint64_t)T * d, 32));
+      LORY_TRY((launch_tc<false, false, 256, MODE_DUALB, EPI_SWIGLU, true, false, 1, 32>("gemm1_swiglu", m_xs, m_xs, m_b1,
+                                                                                         m_b3, m_g, m_u, m_h, p, st)));
+    } else if (use_pairs(T))  // leader loads the Wbar1 rows (G half of the accumulator), its peer the Wbar3 rows (U half)
       LORY_TRY((launch_tc<false, false, 256, MODE_DUALB, EPI_SWIGLU, true, false, 2>("gemm1_swiglu", m_x, m_x, m_b1, m_b3,
                                                                                       m_g, m_u, m_h, p, st)));
     else
@@ -557,7 +563,12 @@ int tc_ffn_forward(const lory_dims& D, const Layout& Lo, char* ws, const bf16* x
     TcGemmParams p = {};
     p.M = T; p.N = d; p.K = f; p.groups = S; p.status = q.status;
     p.residual = residual;
-    if (narrow) {
+    if (narrow && T <= 32 && !residual) {
+      CUtensorMap m_hs;
+      LORY_TRY(make_map(&m_hs, q.H, f, T, S, f, (uint64_t)T * f, 32));
+      LORY_TRY((launch_tc<false, false, 64, MODE_PLAIN, EPI_BF16, true, false, 1, 32>("gemm2", m_hs, m_hs, m_b2, m_b2, m_y,
+                                                                                      m_y, m_y, p, st)));
+    } else if (narrow) {
       if (residual)
         LORY_TRY((launch_tc<false, false, 64, MODE_PLAIN, EPI_BF16_RESADD, true>("gemm2", m_h, m_h, m_b2, m_b2, m_y, m_y,
                                                                                   m_y, p, st)));
