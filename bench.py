@@ -128,9 +128,9 @@ def implementation_bytes_per_step(wl):
 # the digest of the CUDA sources at that time, and a different digest turns the reported traffic into null.
 NCU_TRAFFIC = {
     "C3": {
-        "sources_sha1": "079d4bef069afda6255f129da43b6372d9be0476",
-        "bytes": {"pool_router": 68e6, "merge": 2753e6, "gemm1_swiglu": 2017e6, "gemm2": 965e6, "dh_dswiglu": 1486e6,
-                  "wgrad": 908e6, "stage2": 3229e6, "router_backward": 3e6, "dx": 1875e6},
+        "sources_sha1": "e88f75926891944b49faa2e00cc08aba28a604a2",
+        "bytes": {"pool_router": 68e6, "merge": 2786e6, "gemm1_swiglu": 2016e6, "gemm2": 965e6, "dh_dswiglu": 1487e6,
+                  "wgrad": 908e6, "stage2": 3236e6, "router_backward": 3e6, "dx": 1875e6},
     },
 }
 
