@@ -17,6 +17,8 @@
 // epilogue warps take whole tiles in turn (two per accumulator, one 64-column half each) without exchanging
 // anything (d = 2048, f = 5504: E = 32, S = 16: 1.52 -> 1.17 ms; S = 64: 1.95 -> 1.64 ms; E = 16, S = 64: 1.65 -> 1.54 ms;
 // at S = 128 the doubled MMA count costs more than it saves, so the arrangement above stays there).
+// With 17..64 segments a tile of this arrangement is 192 columns wide (three blocks; block b of a CTA's i-th tile
+// goes to epilogue warp (3 i + b) mod 4): a third fewer MMAs of the first product per byte.
 // Roles: warp 0 TMA, warp 1 issues the first product and owns TMEM, warps 2..5 epilogue, warp 6 issues the second
 // product.  Two issuing threads because with few segments a tile is small (24 KB at S = 64) and the instruction
 // stream of ONE thread issuing both products (12 MMAs with their descriptors, 2 commits, 2 waits) was what a tile
@@ -45,7 +47,8 @@ struct Stage2Maps {
 struct Stage2Params {
   int S, E, Epad16, s_tiles;  // S: segments of this launch (at most 256); s_tiles = ceil(S / 128)
   int seg_base, S_total;      // first segment of this launch; all segments (row count of a dw slab)
-  int rpt_shift;    // 0: a tile is 128 columns of one row; 1: 64 columns of two neighbouring rows
+  int rpt_shift;    // 0: a tile is ncb * 64 columns of one row; 1: 64 columns of two neighbouring rows
+  int ncb;          // 64-column blocks of a tile: 2, or 3 on the fast path with 33..64 segments (fewer MMAs per byte)
   int ctiles[3];    // column tiles per row
   uint32_t cmagic[3];  // ceil(2^32 / ctiles), 0 for ctiles == 1: n / ctiles == __umulhi(n, cmagic) for every tile index n
   int tile_end[3];  // exclusive prefix sums of (rows rounded up to 64) * ctiles
@@ -88,24 +91,26 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = p.tile_end[2];
   const int STAGES = p.stages;
+  const int NCB = p.ncb;   // 64-column blocks per tile (2; 3 on the fast path with 33..64 segments)
   // tile -> (matrix k, row r, first column c0)
   auto decode = [&](int tile, int& k, int& r, int& c0) {
     k = tile < p.tile_end[0] ? 0 : (tile < p.tile_end[1] ? 1 : 2);
     const int local = tile - (k == 0 ? 0 : p.tile_end[k - 1]);
     // local / ctiles[k] without the division (a single tile per row has no 32-bit reciprocal: magic 0)
     r = p.cmagic[k] ? (int)__umulhi((uint32_t)local, p.cmagic[k]) : local;
-    c0 = (local - r * p.ctiles[k]) * (128 >> p.rpt_shift);
+    c0 = (local - r * p.ctiles[k]) * (p.rpt_shift ? 64 : NCB * 64);
     r <<= p.rpt_shift;
   };
   // the two 64-column halves of a tile: columns c0 and c0 + 64 of row r, or (two-row tiles) column c0 of rows r, r + 1
   const int half_col = p.rpt_shift ? 0 : 64, half_row = p.rpt_shift ? 1 : 0;
+  const uint32_t ACC_COLS = (uint32_t)NCB * 64u;   // TMEM columns of one per-tile accumulator
 
   // debug build: a decoded tile against the padded tile grid of its matrix
   auto tile_ok = [&](int k, int r, int c0) {
     if (!dbg::kOn) return true;
     if (k < 0 || k > 2) return false;
     const int tiles_k = p.tile_end[k] - (k ? p.tile_end[k - 1] : 0);
-    return dbg::coord_ok(r, (tiles_k / p.ctiles[k]) << p.rpt_shift) && dbg::inner_ok(c0, p.ctiles[k] * (128 >> p.rpt_shift));
+    return dbg::coord_ok(r, (tiles_k / p.ctiles[k]) << p.rpt_shift) && dbg::inner_ok(c0, p.ctiles[k] * (p.rpt_shift ? 64 : NCB * 64));
   };
 
   if (threadIdx.x == 0) {
@@ -115,7 +120,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
     }
     for (int a = 0; a < NACC; ++a) {
       ptx::mbar_init(&tmem_full_bar[a], 1);
-      ptx::mbar_init(&tmem_empty_bar[a], p.fast ? 64 : 128);   // fast: two warps read an accumulator
+      ptx::mbar_init(&tmem_empty_bar[a], p.fast ? 32 * p.ncb : 128);   // fast: one warp per 64-column block reads it
     }
     ptx::mbar_init(&w_bar, 1);
     ptx::mbar_init(&d2_bar, 1);
@@ -134,7 +139,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_smem;
-  const uint32_t tmem_d2 = tmem_base + NACC * 128;
+  const uint32_t tmem_d2 = tmem_base + NACC * ACC_COLS;
 
   // second product of one stage: dw [s, e] += dWbar [s, p] . W^T [p, e]   (one accumulator per group of 128 segments,
   // resident in TMEM for the whole kernel; with fewer than 128 segments in the box the rows past them hold whatever
@@ -143,10 +148,10 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
   auto issue_second = [&](uint32_t d16, int st, bool first) {
     const uint64_t d2ab = ptx::make_smem_desc(0, 16, 1024);   // K-major tiles; only the 14-bit address varies
     const uint32_t cb16 = (uint32_t)p.cb_stride >> 4, t16 = (uint32_t)(p.Epad16 * 128) >> 4;
-    const uint32_t tb16 = d16 + 2 * cb16;                     // the stage's expert tile
+    const uint32_t tb16 = d16 + (uint32_t)NCB * cb16;         // the stage's expert tile
     const uint32_t tmem_d2s = tmem_d2 + st * p.Epad16;
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
+    for (int j = 0; j < NCB; ++j) {
 #pragma unroll
       for (int k16 = 0; k16 < 4; ++k16) {
         const uint64_t adesc = d2ab | (uint64_t)(d16 + j * cb16 + k16 * 2);
@@ -189,7 +194,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
             abort_flag = 1;
           }
           uint8_t* sD = s_stage + (size_t)s * p.stage_bytes;
-          uint8_t* sT = sD + 2 * p.cb_stride;
+          uint8_t* sT = sD + NCB * p.cb_stride;
           if (!dbg::check(dbg::smem_ok(sD, (uint32_t)p.stage_bytes) && dbg::coord_ok(st, 2), p.status)) continue;
           ptx::mbar_expect_tx(&full_bar[s], tx);
           issued |= 1u << s;
@@ -202,8 +207,8 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           } else {            // one box of two column blocks
             ptx::tma_load_5d(sD, &maps.dwbar[k], &full_bar[s], 0, r & 63, p.seg_base + st * 128, c0 >> 6, r >> 6);
           }
-          ptx::tma_load_3d(sT, &maps.theta[k], &full_bar[s], c0, 0, r);
-          ptx::tma_load_3d(sT + p.Epad16 * 128, &maps.theta[k], &full_bar[s], c0 + half_col, 0, r + half_row);
+          for (int j = 0; j < NCB; ++j)
+            ptx::tma_load_3d(sT + j * p.Epad16 * 128, &maps.theta[k], &full_bar[s], c0 + j * half_col, 0, r + j * half_row);
         }
       }
       if (abort_flag) {
@@ -213,7 +218,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc1 = ptx::make_idesc_bf16(128, 128, true, true);
+      const uint32_t idesc1 = ptx::make_idesc_bf16(128, NCB * 64, true, true);
       if (!ptx::mbar_wait(&w_bar, 0, &abort_flag)) {
         atomicOr(p.status, STATUS_TIMEOUT_MMA);
         abort_flag = 1;
@@ -235,9 +240,9 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
           atomicOr(p.status, STATUS_TIMEOUT_MMA);
           abort_flag = 1;
         }
-        const uint32_t tmem_d1 = tmem_base + acc * 128;
+        const uint32_t tmem_d1 = tmem_base + acc * ACC_COLS;
         // debug build: the per-tile accumulator inside the 512 columns
-        const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d1, tmem_base, 512, 128), p.status);
+        const bool acc_ok = dbg::check(dbg::tmem_ok(tmem_d1, tmem_base, 512, ACC_COLS), p.status);
         for (int st = 0; st < p.s_tiles; ++st, s = (s + 1 == STAGES ? 0 : s + 1), ph ^= (s == 0)) {
           if (!ptx::mbar_wait(&full_bar[s], ph, &abort_flag)) {
             atomicOr(p.status, STATUS_TIMEOUT_MMA);
@@ -311,22 +316,26 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
     const int xlane = p.xch_bytes >> 5, xmask = (xlane >> 4) - 1;
     uint8_t* xch = s_xch + pair * 2 * p.xch_bytes + lane * xlane;
     if (p.fast) {
-      // Every 32-lane quarter of an accumulator holds the finished sums of all (<= 32) experts.  Warps 0, 1 of this
-      // role take the tiles of accumulator 0 (this CTA's even tiles), warps 2, 3 those of accumulator 1, one 64-column
-      // half each: no exchange between warps, and a warp has two tile periods for its load - convert - store chain.
-      const int my_acc = q >> 1, half = q & 1;
+      // Every 32-lane quarter of an accumulator holds the finished sums of all (<= 32) experts, so any warp can take
+      // any 64-column block of any tile from its own lanes.  Block b of this CTA's i-th tile goes to warp
+      // (i * NCB + b) mod 4: with two blocks per tile warps 0, 1 serve the even tiles and 2, 3 the odd ones; with
+      // three, every warp serves three tiles out of four.  No exchange between warps, and a warp has more than a
+      // tile period for its load - convert - store chain.
       wsg.buf = s_out + q * 8192;   // four storing warps: the exchange buffers serve as staging too
-      uint32_t n = 0;
-      for (int tile = blockIdx.x + my_acc * gridDim.x; tile < num_tiles; tile += 2 * gridDim.x, ++n) {
+      uint32_t i = 0;
+      for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++i) {
+        const int half = (int)((q - i * (uint32_t)NCB) & 3u);   // the block of this tile that is this warp's, if < NCB
+        if (half >= NCB) continue;
+        const uint32_t my_acc = i & 1u;
         int k, row, c0;
         decode(tile, k, row, c0);
-        if (!ptx::mbar_wait(&tmem_full_bar[my_acc], n & 1u, &abort_flag)) {
+        if (!ptx::mbar_wait(&tmem_full_bar[my_acc], (i >> 1) & 1u, &abort_flag)) {
           atomicOr(p.status, STATUS_TIMEOUT_EPI);
           abort_flag = 1;
         }
         __syncwarp();  // every lane polls by itself; the warp-wide tcgen05 instructions below need it whole again
         ptx::tc_fence_after_sync();
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + my_acc * 128 + half * 64;
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + my_acc * ACC_COLS + half * 64;
         if (!dbg::check(tile_ok(k, row, c0) && dbg::tmem_ok(taddr, tmem_base, 512, 64) && dbg::smem_ok(wsg.buf, 8192),
                         p.status)) {
           ptx::tc_fence_before_sync();
@@ -378,7 +387,7 @@ stage2_kernel(const __grid_constant__ Stage2Maps maps, const Stage2Params p) {
       }
       __syncwarp();  // every lane polls by itself; the warp-wide tcgen05 instructions below need it whole again
       ptx::tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 128;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * ACC_COLS;
       // debug build: a tile whose coordinates, accumulator columns or staging buffers are out of range is drained
       // (every term is the same for the two warps of a couple, which meet at a named barrier below)
       const bool tile_fine = dbg::check(tile_ok(k, row, c0) && dbg::tmem_ok(taddr, tmem_base, 512, 128) &&

@@ -270,10 +270,11 @@ size_t tc_blocked_elems(const lory_dims& D, int R, int C) {
   return (size_t)((R + 63) / 64) * ((C + 63) / 64) * S * 4096;
 }
 
-// Two-row tiles (64 columns of rows r, r + 1) pay off only with few segments, where the expert traffic dominates
-// (S = 16: 1.67 -> 1.56 ms at d = 2048, f = 5504, E = 32); at S >= 64 they measure the same as 128 columns of one row.
+// Two-row tiles (64 columns of rows r, r + 1) pay off only with very few segments, where the expert traffic dominates
+// (S = 16: 1.67 -> 1.56 ms at d = 2048, f = 5504, E = 32); at S >= 64 they measure the same as 128 columns of one row,
+// and at S = 32 the three-block tiles below are better (1.42 -> 1.34 ms).
 static int stage2_rpt_shift(const lory_dims& D) {
-  return D.B * (D.L / D.T) <= 32 ? 1 : 0;
+  return D.B * (D.L / D.T) <= 16 ? 1 : 0;
 }
 // One of the (up to three) parameter rectangles a launch of the merge adjoint covers: a whole expert matrix, or a
 // sub-rectangle of one whose per-segment gradients sit in a buffer of their own.  R == 0: not part of the launch.
@@ -284,11 +285,20 @@ struct AdjPiece {
   int R, C;
   uint64_t e_stride, row_stride;  // elements between experts / rows of W_k and dW_k
 };
+// Tiles of three 64-column blocks instead of two where both weight halves go through the tensor core (E <= 32,
+// 17..64 segments): the first product then needs its MMAs once per 192 columns instead of once per 128, and the MMA
+// count is what a tile waits for there (d = 2048, f = 5504: E = 16, S = 64: 1.54 -> 1.34 ms; E = 32, S = 64: 1.64 -> 1.58;
+// S = 32: 1.42 -> 1.34).  Four blocks would not fit TMEM beside the double buffering.
+static int stage2_ncb(const lory_dims& D) {
+  const int S = D.B * (D.L / D.T);
+  return (D.E <= 32 && S > 16 && S <= 64) ? 3 : 2;
+}
 static void stage2_tiles(const lory_dims& D, const int R[3], const int C[3], int ctiles[3], int tile_end[3]) {
   const int rsh = stage2_rpt_shift(D);
+  const int width = rsh ? 64 : stage2_ncb(D) * 64;   // columns per tile
   int acc = 0;
   for (int k = 0; k < 3; ++k) {
-    ctiles[k] = C[k] > 0 ? (C[k] + (128 >> rsh) - 1) / (128 >> rsh) : 1;
+    ctiles[k] = C[k] > 0 ? (C[k] + width - 1) / width : 1;
     acc += (((R[k] + 63) / 64 * 64) >> rsh) * ctiles[k];  // whole row blocks: the rows past R[k] read zeros and store nothing
     tile_end[k] = acc;
   }
@@ -440,6 +450,7 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[
   p.dw_partial = q.dw_partial; p.status = q.status;
   p.slab_add = slab_add ? 1 : 0;
   p.rpt_shift = stage2_rpt_shift(D);
+  p.ncb = stage2_ncb(D);
   stage2_tiles(D, R, C, p.ctiles, p.tile_end);
   for (int k = 0; k < 3; ++k)
     p.cmagic[k] = p.ctiles[k] == 1 ? 0u : (uint32_t)(((1ull << 32) + p.ctiles[k] - 1) / p.ctiles[k]);
@@ -462,7 +473,7 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[
   }
   for (int k = 0; k < 3; ++k) {
     const AdjPiece& a = pc[R[k] > 0 ? k : first];  // an absent piece has no tiles; its maps repeat a present one
-    LORY_TRY(make_blocked_map(&maps.dwbar[k], a.dsrc, a.R, a.C, S, 1, seg_box, p.rpt_shift ? 1 : 2, 1));
+    LORY_TRY(make_blocked_map(&maps.dwbar[k], a.dsrc, a.R, a.C, S, 1, seg_box, p.rpt_shift ? 1 : p.ncb, 1));
     LORY_TRY(make_expert_map(&maps.theta[k], a.wsrc, a.R, a.C, E, p.Epad16, a.e_stride, a.row_stride));
     LORY_TRY(make_expert_map(&maps.out[k], a.ddst, a.R, a.C, E, 32, a.e_stride, a.row_stride));
     p.acc_base[k] = a.ddst;
@@ -471,7 +482,7 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[
     p.e_stride[k] = (long)a.e_stride;
     p.row_stride[k] = (long)a.row_stride;
   }
-  p.stage_bytes = 2 * p.cb_stride + 2 * p.Epad16 * 128;  // dWbar tile (two 64-column blocks) + expert tile
+  p.stage_bytes = p.ncb * (p.cb_stride + p.Epad16 * 128);  // dWbar tile (ncb 64-column blocks) + expert tile
   p.tx_bytes = p.stage_bytes;
   p.xch_bytes = p.dup ? 4096 : 8192;
   // w tiles, output staging, lo/hi exchange; and, when the box has fewer than 128 segments, room behind the last
