@@ -128,9 +128,9 @@ def implementation_bytes_per_step(wl):
 # the digest of the CUDA sources at that time, and a different digest turns the reported traffic into null.
 NCU_TRAFFIC = {
     "C3": {
-        "sources_sha1": "e88f75926891944b49faa2e00cc08aba28a604a2",
-        "bytes": {"pool_router": 68e6, "merge": 2786e6, "gemm1_swiglu": 2016e6, "gemm2": 965e6, "dh_dswiglu": 1487e6,
-                  "wgrad": 908e6, "stage2": 3236e6, "router_backward": 3e6, "dx": 1875e6},
+        "sources_sha1": "cebe8cf3fc030c69f7acb3f3be5693b7b1ceb632",
+        "bytes": {"pool_router": 68e6, "merge": 2792e6, "gemm1_swiglu": 2017e6, "gemm2": 964e6, "dh_dswiglu": 1486e6,
+                  "wgrad": 908e6, "stage2": 3238e6, "router_backward": 3e6, "dx": 1875e6},
     },
 }
 

@@ -28,7 +28,8 @@ struct MergeMaps {
 struct MergeParams {
   int S, E, Epad16, s_tiles;  // S: segments of this launch (at most 256); s_tiles = ceil(S / 128)
   int seg_base;               // first segment of this launch (launches cover the segments 256 at a time)
-  int dup;           // S <= 64: the w maps have 64-row boxes and the 64 segments are placed twice (rows 0..63, 64..127)
+  int dup;           // 1 (S <= 64): the w maps have 64-row boxes and the segments are placed twice (rows 0..63, 64..127);
+                     // 2 (S <= 32): 32-row boxes, placed four times
   int rpt_shift;     // log2 of the rows per tile (1, 2 or 4 rows of 256, 128 or 64 columns)
   int ctiles[3];     // column tiles per row
   int tile_end[3];   // exclusive prefix sums of rows_padded * ctiles
@@ -108,9 +109,10 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
     if (lane == 0) {
       ptx::mbar_expect_tx(&w_bar, (uint32_t)p.s_tiles * 32768u);
       if (p.dup) {
-        for (int h = 0; h < 2; ++h) {
-          ptx::tma_load_3d(s_w + h * 8192, &maps.w_hi, &w_bar, 0, 0, 0);
-          ptx::tma_load_3d(s_w + 16384 + h * 8192, &maps.w_lo, &w_bar, 0, 0, 0);
+        const int copies = 2 * p.dup, bytes = 16384 / copies;   // 2 x 64 rows or 4 x 32 rows of 128 bytes
+        for (int h = 0; h < copies; ++h) {
+          ptx::tma_load_3d(s_w + h * bytes, &maps.w_hi, &w_bar, 0, 0, 0);
+          ptx::tma_load_3d(s_w + 16384 + h * bytes, &maps.w_lo, &w_bar, 0, 0, 0);
         }
       } else {
         for (int st = 0; st < p.s_tiles; ++st) {
@@ -192,9 +194,12 @@ __global__ void __launch_bounds__(192, 1) merge_kernel(const __grid_constant__ M
     wsg.buf = s_out + q * 8192;
     wsg.n = 0;
     // S > 64: this warp's accumulator rows are segments q*32 .. q*32+31 and it walks all four 64-column chunks.
-    // S <= 64 (p.dup): rows 64..127 repeat rows 0..63, so warps 0, 1 take chunks 0, 1 and warps 2, 3 chunks 2, 3.
-    const int seg0 = p.dup ? (q & 1) * 32 : q * 32;
-    const int c_begin = p.dup ? (q >> 1) * 2 : 0, c_end = p.dup ? c_begin + 2 : 4;
+    // S <= 64 (p.dup == 1): rows 64..127 repeat rows 0..63, so warps 0, 1 take chunks 0, 1 and warps 2, 3 chunks 2, 3.
+    // S <= 32 (p.dup == 2): every 32-row quarter holds all segments, and warp q takes chunk q alone: four stores per
+    // tile, none of them empty (with two copies half of the eight stores lie past the last segment).
+    const int seg0 = p.dup == 2 ? 0 : (p.dup ? (q & 1) * 32 : q * 32);
+    const int c_begin = p.dup == 2 ? q : (p.dup ? (q >> 1) * 2 : 0);
+    const int c_end = p.dup == 2 ? q + 1 : (p.dup ? c_begin + 2 : 4);
     uint32_t ai = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       int k, r, c0;

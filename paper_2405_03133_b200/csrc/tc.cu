@@ -396,13 +396,14 @@ static int launch_merge(const lory_dims& D, const WsPtrs& q, const bf16* const s
   MergeParams p = {};
   const int S_launch = S < 256 ? S : 256;  // the routing weights of at most 256 segments stay in shared memory
   p.S = S_launch; p.E = E; p.Epad16 = e_pad16(D); p.s_tiles = (S_launch + 127) / 128; p.status = q.status;
-  p.dup = S <= 64 ? 1 : 0;
+  p.dup = S <= 32 ? 2 : (S <= 64 ? 1 : 0);
   // Tiles of 4 rows x 64 columns: a segment's four 128-byte output pieces of one tile are neighbours in its 64 x 64
   // block (512 contiguous bytes).  Measured against 1 x 256 and 2 x 128: C3 0.546 / 0.520 / 0.524 ms (1, 2, 4 rows),
   // C4 1.064 / 1.036 / 0.996 ms.
   p.rpt_shift = 2;
-  LORY_TRY(make_map(&maps.w_hi, q.w_hi, Ep, S, 1, Ep, 0, p.dup ? 64 : 128));
-  LORY_TRY(make_map(&maps.w_lo, q.w_lo, Ep, S, 1, Ep, 0, p.dup ? 64 : 128));
+  const uint32_t w_box = p.dup == 2 ? 32u : (p.dup ? 64u : 128u);
+  LORY_TRY(make_map(&maps.w_hi, q.w_hi, Ep, S, 1, Ep, 0, w_box));
+  LORY_TRY(make_map(&maps.w_lo, q.w_lo, Ep, S, 1, Ep, 0, w_box));
   int acc = 0;
   for (int k = 0; k < 3; ++k) {
     LORY_TRY(make_expert_map(&maps.theta[k], src[k], R[k], C[k], E, p.Epad16));
@@ -475,7 +476,7 @@ static int launch_stage2(const lory_dims& D, const WsPtrs& q, const AdjPiece pc[
     const AdjPiece& a = pc[R[k] > 0 ? k : first];  // an absent piece has no tiles; its maps repeat a present one
     LORY_TRY(make_blocked_map(&maps.dwbar[k], a.dsrc, a.R, a.C, S, 1, seg_box, p.rpt_shift ? 1 : p.ncb, 1));
     LORY_TRY(make_expert_map(&maps.theta[k], a.wsrc, a.R, a.C, E, p.Epad16, a.e_stride, a.row_stride));
-    LORY_TRY(make_expert_map(&maps.out[k], a.ddst, a.R, a.C, E, 32, a.e_stride, a.row_stride));
+    LORY_TRY(make_expert_map(&maps.out[k], a.ddst, a.R, a.C, E, E < 32 ? (uint32_t)E : 32u, a.e_stride, a.row_stride));  // no box rows past the experts
     p.acc_base[k] = a.ddst;
     p.rows[k] = a.R;
     p.cols[k] = a.C;
